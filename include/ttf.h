@@ -1,0 +1,129 @@
+/*
+ * ttf.h : C ABI of the B200 Temporal Token Fusion library (libttf_b200.so).
+ *
+ * The library implements the pre-LLM pass of Temporal Token Fusion (arXiv 2605.07355, Sec. 3) for one clip
+ * of visual tokens X[F, H, W, C] on one sm_100a GPU:
+ *
+ *   anchor frame a* (Eq. auto_anchor)  ->  best cosine match of every source token inside the
+ *   (2r+1) x (2r+1) window of the anchor grid (Eqs. pi, argmax, dst)  ->  gate keep = 1[s_hat <= t]
+ *   (Eq. gating)  ->  compressed sequence X' = N anchor rows followed by the P preserved source rows
+ *   (Eq. xprime_stack) with their original (k, y, x) position triples (Eqs. mask, compress_pos) and the
+ *   compressed length L' = N + P that prefill and decoding use as position base (Eqs. Lpre, decode_pos).
+ *
+ * Fusion is the paper's identity replacement (Sec. 3, Threshold Gating): a fused token is dropped and the
+ * anchor row dst(k,i) stands for it unchanged; output rows are bit copies of input rows.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer on the current CUDA device unless its name ends in _host.
+ *   - The caller owns every buffer.  The library never frees caller memory and writes at most
+ *     F*H*W rows into out_tokens / out_pos_thw (the worst case, nothing fused).
+ *   - Calls only enqueue work on `stream` (a cudaStream_t passed as an opaque pointer; NULL = legacy default
+ *     stream) and return without synchronising, except the *_host entry point.
+ *   - features: contiguous [F, H, W, C], C fastest, row = one token; dtype selects fp32 or bf16.
+ *     Any C >= 1 is accepted; rows whose byte length is a multiple of 16 with a 16-byte aligned base take
+ *     the vectorised kernels, everything else a scalar path with identical results.
+ *   - r >= 0 is the search radius (window side 2r+1); t is any finite float (not restricted to (0,1)).
+ *   - Return value: a ttf_status.  Host-detectable problems (NULL pointer, non-positive size, negative r,
+ *     non-finite t, unknown dtype, F*H*W*C overflow, workspace too small or misaligned) are reported
+ *     before anything is launched, and nothing is written.  CUDA launch failures return TTF_ERR_CUDA.
+ *   - Similarities are computed in fp32 (bf16 products are exact in fp32; fp32 accumulation); norms are
+ *     floored at 1e-12, so an all-zero token has similarity 0 to everything.  A token is fused iff
+ *     s_hat > t strictly; equal candidates resolve to the lowest anchor index, equal anchor cosines to the
+ *     lowest frame.
+ *   - Results are deterministic: no floating-point atomics, every reduction has a fixed order.
+ *   - The library has no CPU fallback: without a CUDA device every compute entry point fails.
+ */
+#ifndef TTF_B200_H_
+#define TTF_B200_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { TTF_DTYPE_F32 = 0, TTF_DTYPE_BF16 = 1 } ttf_dtype;
+
+typedef enum {
+    TTF_OK = 0,
+    TTF_ERR_INVALID_ARG = 1,   /* NULL pointer, size < 1, r < 0, non-finite t, unknown dtype or option       */
+    TTF_ERR_UNSUPPORTED = 2,   /* sizes beyond int32 indexing (F*H*W >= 2^31 or F*H*W*C*itemsize >= 2^46)    */
+    TTF_ERR_WORKSPACE = 3,     /* caller workspace NULL, smaller than ttf_workspace_bytes or not 256-aligned */
+    TTF_ERR_CUDA = 4           /* a CUDA runtime call failed (see ttf_last_cuda_error)                       */
+} ttf_status;
+
+typedef struct CUstream_st* ttf_stream_t;      /* same type as cudaStream_t */
+
+/* Human-readable name of a ttf_status. Never NULL. */
+const char* ttf_status_string(int status);
+
+/* cudaError_t of the most recent failing CUDA call made by this library on the calling thread (0 if none). */
+int ttf_last_cuda_error(void);
+
+/*
+ * Scratch bytes one call needs for a clip of this shape (per-token inverse norms, per-frame channel sums,
+ * anchor cosines, s_hat / dst / keep, per-frame survivor counts).  Sec. 3 has no counterpart: this is
+ * bookkeeping of the implementation.  The result is a multiple of 256.
+ */
+int ttf_workspace_bytes(int F, int H, int W, int C, int r, int dtype, size_t* bytes);
+
+/*
+ * The whole pass for one clip (Sec. 3; Fig. 1): anchor selection, windowed matching, gating, compaction and
+ * positional alignment.
+ *   out_tokens   [capacity F*H*W rows, C] same dtype as features; rows [0, N) are the anchor frame's tokens,
+ *                rows [N, N+P) the preserved source tokens in ascending flat index k*N + i (Eq. xprime_stack).
+ *   out_count    one int32: L' = N + P (Eq. Lpre).  pos_dec(l) = L' + T + l (Eq. decode_pos) is
+ *                ttf_decode_pos below.
+ *   out_pos_thw  [capacity F*H*W, 3] int32; row j = (k, y, x) of output row j (Eq. compress_pos).
+ * Rows beyond L' are not written.  Scratch comes from a cache the library keeps per (device, stream),
+ * allocated with cudaMalloc on first use and grown when a larger clip arrives; two calls on the same stream
+ * are ordered by the stream, calls on different streams use different scratch.
+ */
+int ttf_compress(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                 void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream);
+
+/* Same, with caller-owned scratch: `workspace` must be 256-byte aligned device memory of at least
+ * ttf_workspace_bytes(...) bytes that no other in-flight call uses.  Allocates nothing. */
+int ttf_compress_ws(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                    void* out_tokens, int* out_count, int* out_pos_thw,
+                    void* workspace, size_t workspace_bytes, ttf_stream_t stream);
+
+/*
+ * Query: the pass stopped before compaction (Sec. 3, Anchor Frame Selection to Threshold Gating).
+ * Any output pointer may be NULL.
+ *   out_anchor    one int32: a* (Eq. auto_anchor)
+ *   out_keep      [F*H*W] uint8: retention mask m_{k,i} (Eq. mask); the anchor frame is all 1
+ *   out_dst       [F*H*W] int32: dst(k,i), anchor-frame cell index in [0, N) (Eq. dst); i for anchor rows
+ *   out_best_sim  [F*H*W] fp32: s_hat_{k,i} (Eq. argmax); 1 for anchor rows
+ *   out_fuse_cnt  [H*W] int32: number of source tokens fused into each anchor cell
+ *                 (|{(k,i): m_{k,i} = 0, dst(k,i) = j}|, the bookkeeping side of identity replacement)
+ */
+int ttf_query(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+              int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
+              int* out_fuse_cnt, ttf_stream_t stream);
+
+int ttf_query_ws(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                 int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
+                 int* out_fuse_cnt, void* workspace, size_t workspace_bytes, ttf_stream_t stream);
+
+/*
+ * The same pass for callers whose tensors live in HOST memory (all four pointers are host pointers; pinned
+ * memory makes the copies asynchronous).  Copies features to the device, runs ttf_compress, copies L' and the
+ * first L' rows of tokens and positions back, and returns after synchronising.  Device staging buffers are
+ * cached per device and reused.  out_count_host receives L'.
+ */
+int ttf_compress_host(const void* features_host, int F, int H, int W, int C, int r, float t, int dtype,
+                      void* out_tokens_host, int* out_count_host, int* out_pos_thw_host);
+
+/* Frees every cached scratch / staging buffer of the calling process (all devices).  Synchronises. */
+int ttf_release(void);
+
+/* Eqs. (Lpre), (decode_pos): position of the l-th generated token after a prefill of L' visual tokens
+ * and T text tokens. */
+static inline long long ttf_decode_pos(long long L_prime, long long T, long long l) { return L_prime + T + l; }
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TTF_B200_H_ */

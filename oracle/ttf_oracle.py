@@ -1,0 +1,179 @@
+"""ctypes front end of the CPU oracle (oracle/ttf_oracle.c).  TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the CPU-baseline leg of the benchmark may import this module; the CUDA
+library never does.  This file only marshals arrays: every step of the method is in the C file, which
+follows Sec. 3 of the paper (anchor rule, local-window matching, threshold gate, compaction, positions).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ttf_oracle.c")
+_LIB = os.path.join(_HERE, "libttf_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no fast-math, so double arithmetic stays in source order)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-fopenmp", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        c_int, c_sz, vp = ctypes.c_int, ctypes.c_size_t, ctypes.c_void_p
+        lib.ttf_oracle_threads.restype = c_int
+        lib.ttf_oracle_anchor.restype = c_int
+        lib.ttf_oracle_anchor.argtypes = [vp, c_int, c_int, c_int, vp]
+        lib.ttf_oracle_match.restype = None
+        lib.ttf_oracle_match.argtypes = [vp, c_int, c_int, c_int, c_int, c_int, c_int, vp, vp, vp]
+        lib.ttf_oracle_match_global.restype = None
+        lib.ttf_oracle_match_global.argtypes = [vp, c_int, c_int, c_int, c_int, vp, vp]
+        lib.ttf_oracle_gate.restype = None
+        lib.ttf_oracle_gate.argtypes = [vp, c_int, c_int, c_int, ctypes.c_float, vp]
+        lib.ttf_oracle_fuse_count.restype = None
+        lib.ttf_oracle_fuse_count.argtypes = [vp, vp, c_int, c_int, c_int, vp]
+        lib.ttf_oracle_compact.restype = c_int
+        lib.ttf_oracle_compact.argtypes = [vp, c_sz, vp, c_int, c_int, c_int, c_int, vp, vp, vp]
+        lib.ttf_oracle_decode_pos.restype = ctypes.c_longlong
+        lib.ttf_oracle_decode_pos.argtypes = [ctypes.c_longlong] * 3
+        _lib = lib
+    return _lib
+
+
+def threads() -> int:
+    return int(_load().ttf_oracle_threads())
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _widen(X: np.ndarray) -> np.ndarray:
+    """fp32 view of the clip: fp32 as is, bf16 bit patterns (uint16) widened exactly (16-bit shift)."""
+    if X.dtype == np.float32:
+        return np.ascontiguousarray(X)
+    if X.dtype == np.uint16:
+        return (np.ascontiguousarray(X).astype(np.uint32) << np.uint32(16)).view(np.float32)
+    raise TypeError("clip must be float32 or uint16 (bf16 bit patterns)")
+
+
+def _shape(X: np.ndarray):
+    if X.ndim != 4:
+        raise ValueError("clip must be [F, H, W, C]")
+    return X.shape
+
+
+def anchor(X: np.ndarray):
+    """Eq. (auto_anchor): returns (a*, cos[F])."""
+    F, H, W, C = _shape(X)
+    Xf = _widen(X)
+    cos = np.empty(F, dtype=np.float64)
+    a = _load().ttf_oracle_anchor(_ptr(Xf), F, H * W, C, _ptr(cos))
+    return int(a), cos
+
+
+def match(X: np.ndarray, r: int, a: int):
+    """Eqs. (pi), (argmax), (dst): returns (s_hat[F*N] f64, dst[F*N] i32, second[F*N] f64)."""
+    F, H, W, C = _shape(X)
+    Xf = _widen(X)
+    n = F * H * W
+    s_hat = np.empty(n, dtype=np.float64)
+    dst = np.empty(n, dtype=np.int32)
+    second = np.empty(n, dtype=np.float64)
+    _load().ttf_oracle_match(_ptr(Xf), F, H, W, C, int(r), int(a), _ptr(s_hat), _ptr(dst), _ptr(second))
+    return s_hat, dst, second
+
+
+def match_global(X: np.ndarray, a: int):
+    """Best cosine over ALL anchor tokens (all-pairs search); cross-check only."""
+    F, H, W, C = _shape(X)
+    Xf = _widen(X)
+    n = F * H * W
+    s_hat = np.empty(n, dtype=np.float64)
+    dst = np.empty(n, dtype=np.int32)
+    _load().ttf_oracle_match_global(_ptr(Xf), F, H * W, C, int(a), _ptr(s_hat), _ptr(dst))
+    return s_hat, dst
+
+
+def gate(s_hat: np.ndarray, F: int, N: int, a: int, t: float) -> np.ndarray:
+    """Eqs. (gating), (mask): keep[F*N] uint8."""
+    s_hat = np.ascontiguousarray(s_hat, dtype=np.float64)
+    keep = np.empty(F * N, dtype=np.uint8)
+    _load().ttf_oracle_gate(_ptr(s_hat), F, N, int(a), float(t), _ptr(keep))
+    return keep
+
+
+def fuse_count(keep: np.ndarray, dst: np.ndarray, F: int, N: int, a: int) -> np.ndarray:
+    keep = np.ascontiguousarray(keep, dtype=np.uint8)
+    dst = np.ascontiguousarray(dst, dtype=np.int32)
+    out = np.empty(N, dtype=np.int32)
+    _load().ttf_oracle_fuse_count(_ptr(keep), _ptr(dst), F, N, int(a), _ptr(out))
+    return out
+
+
+def compact(X: np.ndarray, keep: np.ndarray, a: int):
+    """Eqs. (xprime_stack), (compress_pos): returns (tokens[L', C] same dtype as X, pos[L', 3] i32,
+    index[L'] i32 flat source index of each output row, L')."""
+    F, H, W, C = _shape(X)
+    Xc = np.ascontiguousarray(X)
+    keep = np.ascontiguousarray(keep, dtype=np.uint8)
+    n = F * H * W
+    tokens = np.empty((n, C), dtype=X.dtype)
+    pos = np.empty((n, 3), dtype=np.int32)
+    index = np.empty(n, dtype=np.int32)
+    L = _load().ttf_oracle_compact(_ptr(Xc), C * X.dtype.itemsize, _ptr(keep), F, H, W, int(a),
+                                   _ptr(tokens), _ptr(pos), _ptr(index))
+    return tokens[:L], pos[:L], index[:L], int(L)
+
+
+def decode_pos(L_prime: int, T: int, l: int) -> int:
+    """Eqs. (Lpre), (decode_pos)."""
+    return int(_load().ttf_oracle_decode_pos(L_prime, T, l))
+
+
+@dataclass
+class OracleResult:
+    anchor: int
+    anchor_cos: np.ndarray      # [F] f64
+    s_hat: np.ndarray           # [F*N] f64
+    dst: np.ndarray             # [F*N] i32
+    second: np.ndarray          # [F*N] f64 runner-up similarity
+    keep: np.ndarray            # [F*N] u8
+    fuse_cnt: np.ndarray        # [N] i32
+    tokens: np.ndarray          # [L', C]
+    pos: np.ndarray             # [L', 3] i32
+    index: np.ndarray           # [L'] i32
+    count: int                  # L' = N + P
+
+    @property
+    def rho(self) -> float:
+        return 1.0 - self.count / float(self.keep.size)
+
+
+def compress(X: np.ndarray, r: int, t: float, anchor_frame: Optional[int] = None,
+             forced_keep: Optional[np.ndarray] = None) -> OracleResult:
+    """The whole pass in the paper's order.  ``anchor_frame`` overrides the anchor rule (first / last /
+    explicit anchors of Table 1); ``forced_keep`` replaces the gate's decisions (used after near-threshold
+    differences have been accepted, so that counts, positions and rows can still be compared exactly)."""
+    F, H, W, C = _shape(X)
+    N = H * W
+    a_auto, cos = anchor(X)
+    a = a_auto if anchor_frame is None else int(anchor_frame)
+    s_hat, dst, second = match(X, r, a)
+    keep = gate(s_hat, F, N, a, t) if forced_keep is None else np.ascontiguousarray(forced_keep, dtype=np.uint8).reshape(-1)
+    fc = fuse_count(keep, dst, F, N, a)
+    tokens, pos, index, L = compact(X, keep, a)
+    return OracleResult(a, cos, s_hat, dst, second, keep, fc, tokens, pos, index, L)
