@@ -1,0 +1,189 @@
+"""Thin Python binding of libttf_b200.so: argument marshalling only.
+
+Function names and argument order follow include/ttf.h.  Tensors are torch tensors (device memory and
+streams come from PyTorch); every step of the pass runs in the library's CUDA kernels.  There is no CPU
+fallback: if the shared library is missing or no CUDA device is present the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libttf_b200.so")
+
+TTF_DTYPE_F32, TTF_DTYPE_BF16 = 0, 1
+TTF_OK = 0
+
+EXPORTS = [
+    "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
+    "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release",
+]
+
+_lib = None
+
+
+class TTFError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        name = lib().ttf_status_string(status).decode()
+        extra = f" (cudaError {lib().ttf_last_cuda_error()})" if name == "TTF_ERR_CUDA" else ""
+        super().__init__(f"{where}: {name}{extra}")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads the C-ABI library (built by paper_2605_07355_b200.build); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(
+                f"{LIB_PATH} not found: build it with `python -m paper_2605_07355_b200.build` (needs nvcc)")
+        L = ctypes.CDLL(LIB_PATH)
+        i, f, vp, sz = ctypes.c_int, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t
+        shape = [i, i, i, i, i]                       # F, H, W, C, r
+        L.ttf_status_string.restype = ctypes.c_char_p
+        L.ttf_status_string.argtypes = [i]
+        L.ttf_last_cuda_error.restype = i
+        L.ttf_last_cuda_error.argtypes = []
+        L.ttf_workspace_bytes.restype = i
+        L.ttf_workspace_bytes.argtypes = shape + [i, ctypes.POINTER(sz)]
+        L.ttf_compress.restype = i
+        L.ttf_compress.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp]
+        L.ttf_compress_ws.restype = i
+        L.ttf_compress_ws.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, sz, vp]
+        L.ttf_query.restype = i
+        L.ttf_query.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp]
+        L.ttf_query_ws.restype = i
+        L.ttf_query_ws.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.ttf_compress_host.restype = i
+        L.ttf_compress_host.argtypes = [vp] + shape + [f, i, vp, vp, vp]
+        L.ttf_release.restype = i
+        L.ttf_release.argtypes = []
+        _lib = L
+    return _lib
+
+
+def _dtype_code(x: torch.Tensor) -> int:
+    if x.dtype == torch.float32:
+        return TTF_DTYPE_F32
+    if x.dtype == torch.bfloat16:
+        return TTF_DTYPE_BF16
+    raise TypeError(f"features must be float32 or bfloat16, got {x.dtype}")
+
+
+def _check_features(x: torch.Tensor, device: str):
+    if x.dim() != 4:
+        raise ValueError("features must be [F, H, W, C]")
+    if not x.is_contiguous():
+        raise ValueError("features must be contiguous")
+    if device == "cuda" and not x.is_cuda:
+        raise ValueError("features must be a CUDA tensor")
+    if device == "cpu" and x.is_cuda:
+        raise ValueError("features must be a host tensor")
+    return tuple(int(v) for v in x.shape)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _p(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def ttf_workspace_bytes(F: int, H: int, W: int, C: int, r: int, dtype: int) -> int:
+    n = ctypes.c_size_t(0)
+    rc = lib().ttf_workspace_bytes(F, H, W, C, r, dtype, ctypes.byref(n))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_workspace_bytes")
+    return int(n.value)
+
+
+def ttf_compress(features: torch.Tensor, r: int, t: float, out_tokens: Optional[torch.Tensor] = None,
+                 out_count: Optional[torch.Tensor] = None, out_pos_thw: Optional[torch.Tensor] = None,
+                 workspace: Optional[torch.Tensor] = None, stream=None):
+    """ttf_compress / ttf_compress_ws.  Returns (out_tokens [F*H*W, C], out_count int32[1],
+    out_pos_thw int32 [F*H*W, 3]); only the first out_count rows are defined.  Does not synchronise."""
+    F, H, W, C = _check_features(features, "cuda")
+    dev = features.device
+    n = F * H * W
+    if out_tokens is None:
+        out_tokens = torch.empty((n, C), dtype=features.dtype, device=dev)
+    if out_count is None:
+        out_count = torch.empty(1, dtype=torch.int32, device=dev)
+    if out_pos_thw is None:
+        out_pos_thw = torch.empty((n, 3), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        sp = _stream_ptr(stream)
+        if workspace is None:
+            rc = lib().ttf_compress(_p(features), F, H, W, C, int(r), float(t), _dtype_code(features),
+                                    _p(out_tokens), _p(out_count), _p(out_pos_thw), sp)
+        else:
+            rc = lib().ttf_compress_ws(_p(features), F, H, W, C, int(r), float(t), _dtype_code(features),
+                                       _p(out_tokens), _p(out_count), _p(out_pos_thw),
+                                       _p(workspace), workspace.numel() * workspace.element_size(), sp)
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_compress")
+    return out_tokens, out_count, out_pos_thw
+
+
+def ttf_query(features: torch.Tensor, r: int, t: float, workspace: Optional[torch.Tensor] = None, stream=None,
+              want=("anchor", "keep", "dst", "best_sim", "fuse_cnt")) -> dict:
+    """ttf_query / ttf_query_ws.  Returns the requested device tensors.  Does not synchronise."""
+    F, H, W, C = _check_features(features, "cuda")
+    dev = features.device
+    n = F * H * W
+    out = {
+        "anchor": torch.empty(1, dtype=torch.int32, device=dev) if "anchor" in want else None,
+        "keep": torch.empty(n, dtype=torch.uint8, device=dev) if "keep" in want else None,
+        "dst": torch.empty(n, dtype=torch.int32, device=dev) if "dst" in want else None,
+        "best_sim": torch.empty(n, dtype=torch.float32, device=dev) if "best_sim" in want else None,
+        "fuse_cnt": torch.empty(H * W, dtype=torch.int32, device=dev) if "fuse_cnt" in want else None,
+    }
+    args = [_p(features), F, H, W, C, int(r), float(t), _dtype_code(features), _p(out["anchor"]), _p(out["keep"]),
+            _p(out["dst"]), _p(out["best_sim"]), _p(out["fuse_cnt"])]
+    with torch.cuda.device(dev):
+        sp = _stream_ptr(stream)
+        if workspace is None:
+            rc = lib().ttf_query(*args, sp)
+        else:
+            rc = lib().ttf_query_ws(*args, _p(workspace), workspace.numel() * workspace.element_size(), sp)
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_query")
+    return {k: v for k, v in out.items() if v is not None}
+
+
+def ttf_compress_host(features: torch.Tensor, r: int, t: float, out_tokens: Optional[torch.Tensor] = None,
+                      out_pos_thw: Optional[torch.Tensor] = None, device: Optional[int] = None):
+    """ttf_compress_host: HOST tensors in and out (pinned memory recommended).  Returns
+    (out_tokens[:L'], L', out_pos_thw[:L']); synchronous."""
+    F, H, W, C = _check_features(features, "cpu")
+    n = F * H * W
+    if out_tokens is None:
+        out_tokens = torch.empty((n, C), dtype=features.dtype)
+    if out_pos_thw is None:
+        out_pos_thw = torch.empty((n, 3), dtype=torch.int32)
+    cnt = ctypes.c_int(0)
+    with torch.cuda.device(torch.cuda.current_device() if device is None else device):
+        rc = lib().ttf_compress_host(_p(features), F, H, W, C, int(r), float(t), _dtype_code(features),
+                                     _p(out_tokens), ctypes.cast(ctypes.byref(cnt), ctypes.c_void_p), _p(out_pos_thw))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_compress_host")
+    L = int(cnt.value)
+    return out_tokens[:L], L, out_pos_thw[:L]
+
+
+def ttf_release() -> None:
+    rc = lib().ttf_release()
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_release")
+
+
+def ttf_decode_pos(L_prime: int, T: int, l: int) -> int:
+    """Eqs. (Lpre), (decode_pos): the inline helper of ttf.h."""
+    return int(L_prime) + int(T) + int(l)

@@ -174,7 +174,7 @@ _LITERAL = [
 ]
 
 # s0 values written by oracle/calibrate_clips.py (rho(t=0.70) = 0.67 +- 0.01 on the seeds above)
-_S0 = {"tiny": 0.4575, "vl2b": 0.4004, "vl8b": 0.3547, "long": 0.2976, "wide": 0.35}
+_S0 = {"tiny": 0.4575, "vl2b": 0.4004, "vl8b": 0.3547, "long": 0.317, "wide": 0.2861}
 _HETERO = 0.8
 
 

@@ -1,0 +1,334 @@
+// C ABI of libttf_b200.so: argument validation, scratch management and the launch sequence of one clip.
+// Declarations and the contract of every entry point are in include/ttf.h.
+#include "../../include/ttf.h"
+#include "ttf_internal.cuh"
+
+#include <cmath>
+#include <map>
+#include <mutex>
+#include <utility>
+#include <vector>
+
+namespace ttf {
+
+static thread_local int tl_cuda_error = 0;
+
+static int cuda_fail(cudaError_t e) {
+    tl_cuda_error = (int)e;
+    return TTF_ERR_CUDA;
+}
+
+int sm_count() {
+    static std::mutex mu;
+    static std::map<int, int> cache;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = cache.find(dev);
+    if (it != cache.end()) return it->second;
+    int n = 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    cache[dev] = n;
+    return n;
+}
+
+static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+void carve_scratch(const Problem& p, void* base, Scratch* s) {
+    size_t off = 0;
+    char* b = reinterpret_cast<char*>(base);
+    auto take = [&](size_t bytes) { size_t o = off; off = align256(off + bytes); return b ? (void*)(b + o) : nullptr; };
+    const size_t FN = (size_t)p.F * p.N;
+    s->hdr = (int*)take(sizeof(int) * kHdrInts);
+    s->cnt = (int*)take(sizeof(int) * p.F);
+    s->prefix = (int*)take(sizeof(int) * ((size_t)p.F + 1));
+    s->fcos = (float*)take(sizeof(float) * p.F);
+    s->g = (float*)take(sizeof(float) * p.C);
+    s->S = (float*)take(sizeof(float) * (size_t)p.F * p.C);
+    s->ssq = (float*)take(sizeof(float) * (size_t)p.nslice * FN);
+    s->shat = (float*)take(sizeof(float) * FN);
+    s->dst = (int*)take(sizeof(int) * FN);
+    s->keep = (unsigned char*)take(FN);
+    s->fuse_cnt = (int*)take(sizeof(int) * p.N);
+    s->bytes = off;
+}
+
+// Validates the shape arguments and fills the derived fields.  Pointers are checked by the callers.
+static int make_problem(const void* X, int F, int H, int W, int C, int r, float t, int dtype, Problem* p) {
+    if (F < 1 || H < 1 || W < 1 || C < 1 || r < 0) return TTF_ERR_INVALID_ARG;
+    if (dtype != TTF_DTYPE_F32 && dtype != TTF_DTYPE_BF16) return TTF_ERR_INVALID_ARG;
+    if (!std::isfinite(t)) return TTF_ERR_INVALID_ARG;
+    const long long N = (long long)H * W;
+    const long long FN = N * F;
+    if (N >= (1LL << 31) || FN >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
+    const long long esize = dtype == TTF_DTYPE_F32 ? 4 : 2;
+    if ((double)FN * (double)C * (double)esize >= (double)(1LL << 46)) return TTF_ERR_UNSUPPORTED;
+    p->X = X; p->F = F; p->H = H; p->W = W; p->C = C; p->r = r; p->t = t; p->dtype = dtype;
+    p->N = (int)N;
+    const long long row_bytes = (long long)C * esize;
+    p->vec = (row_bytes % 16 == 0) && (reinterpret_cast<uintptr_t>(X) % 16 == 0);
+    p->lanes_elems = p->vec ? (int)(16 / esize) : 1;
+    const long long per_slice = 32LL * p->lanes_elems;
+    p->nslice = (int)((C + per_slice - 1) / per_slice);
+    if ((long long)F * p->nslice >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
+    p->anchor_mode = 0; p->anchor_arg = 0;
+    return TTF_OK;
+}
+
+// ---- scratch cache: one block per (device, stream), grown on demand -------------------------------------
+struct CacheEntry { void* ptr = nullptr; size_t bytes = 0; };
+static std::mutex g_mu;
+static std::map<std::pair<int, cudaStream_t>, CacheEntry> g_scratch;
+
+static int cached_scratch(size_t bytes, cudaStream_t st, void** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    std::lock_guard<std::mutex> lk(g_mu);
+    CacheEntry& ce = g_scratch[std::make_pair(dev, st)];
+    if (ce.bytes < bytes) {
+        if (ce.ptr) {
+            // earlier calls on this stream may still read the old block
+            e = cudaStreamSynchronize(st);
+            if (e != cudaSuccess) return cuda_fail(e);
+            cudaFree(ce.ptr);
+            ce.ptr = nullptr; ce.bytes = 0;
+        }
+        e = cudaMalloc(&ce.ptr, bytes);
+        if (e != cudaSuccess) { ce.ptr = nullptr; return cuda_fail(e); }
+        ce.bytes = bytes;
+    }
+    *out = ce.ptr;
+    return TTF_OK;
+}
+
+static int check_ws(const Problem& p, void* ws, size_t ws_bytes, Scratch* s) {
+    carve_scratch(p, nullptr, s);
+    if (!ws || ws_bytes < s->bytes || reinterpret_cast<uintptr_t>(ws) % 256 != 0) return TTF_ERR_WORKSPACE;
+    carve_scratch(p, ws, s);
+    return TTF_OK;
+}
+
+// steps shared by compress and query: norms + frame sums, anchor, matching + gate
+static int run_front(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
+                     unsigned char* keep, cudaStream_t st) {
+    cudaError_t e = launch_norm_sum(p, s, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_anchor_pick(p, s, out_anchor, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = launch_match(p, s, shat, dst, keep, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return TTF_OK;
+}
+
+static int compress_impl(const Problem& p, void* ws, void* out_tokens, int* out_count, int* out_pos,
+                         cudaStream_t st) {
+    Scratch s;
+    carve_scratch(p, ws, &s);
+    int rc = run_front(p, s, nullptr, s.shat, s.dst, s.keep, st);
+    if (rc != TTF_OK) return rc;
+    cudaError_t e = launch_compact(p, s, out_tokens, out_pos, out_count, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return TTF_OK;
+}
+
+static int query_impl(const Problem& p, void* ws, int* out_anchor, unsigned char* out_keep, int* out_dst,
+                      float* out_sim, int* out_fuse, cudaStream_t st) {
+    Scratch s;
+    carve_scratch(p, ws, &s);
+    float* shat = out_sim ? out_sim : s.shat;
+    int* dst = out_dst ? out_dst : s.dst;
+    unsigned char* keep = out_keep ? out_keep : s.keep;
+    int rc = run_front(p, s, out_anchor, shat, dst, keep, st);
+    if (rc != TTF_OK) return rc;
+    if (out_fuse) {
+        cudaError_t e = launch_fuse_count(p, s, dst, keep, out_fuse, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return TTF_OK;
+}
+
+// ---- host-buffer entry point: staging buffers per device -------------------------------------------------
+struct Staging {
+    void* feat = nullptr; size_t feat_bytes = 0;
+    void* tok = nullptr; size_t tok_bytes = 0;
+    int* pos = nullptr; size_t pos_bytes = 0;
+    int* count = nullptr;
+    cudaStream_t stream = nullptr;
+};
+static std::map<int, Staging> g_staging;
+
+static cudaError_t grow(void** p, size_t* have, size_t want) {
+    if (*have >= want) return cudaSuccess;
+    if (*p) cudaFree(*p);
+    *p = nullptr; *have = 0;
+    cudaError_t e = cudaMalloc(p, want);
+    if (e == cudaSuccess) *have = want;
+    return e;
+}
+
+}  // namespace ttf
+
+using namespace ttf;
+
+extern "C" {
+
+const char* ttf_status_string(int status) {
+    switch (status) {
+        case TTF_OK: return "TTF_OK";
+        case TTF_ERR_INVALID_ARG: return "TTF_ERR_INVALID_ARG";
+        case TTF_ERR_UNSUPPORTED: return "TTF_ERR_UNSUPPORTED";
+        case TTF_ERR_WORKSPACE: return "TTF_ERR_WORKSPACE";
+        case TTF_ERR_CUDA: return "TTF_ERR_CUDA";
+        default: return "TTF_ERR_UNKNOWN";
+    }
+}
+
+int ttf_last_cuda_error(void) { return tl_cuda_error; }
+
+int ttf_workspace_bytes(int F, int H, int W, int C, int r, int dtype, size_t* bytes) {
+    if (!bytes) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    // the scalar layout (one channel per lane) is the larger one: size for it so that the same scratch
+    // serves a clip whatever the alignment of its base pointer
+    int rc = make_problem(reinterpret_cast<const void*>(uintptr_t(1)), F, H, W, C, r, 0.f, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    Scratch s;
+    carve_scratch(p, nullptr, &s);
+    *bytes = s.bytes;
+    return TTF_OK;
+}
+
+int ttf_compress_ws(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                    void* out_tokens, int* out_count, int* out_pos_thw,
+                    void* workspace, size_t workspace_bytes, ttf_stream_t stream) {
+    if (!features || !out_tokens || !out_count || !out_pos_thw) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    Scratch s;
+    rc = check_ws(p, workspace, workspace_bytes, &s);
+    if (rc != TTF_OK) return rc;
+    return compress_impl(p, workspace, out_tokens, out_count, out_pos_thw, (cudaStream_t)stream);
+}
+
+int ttf_compress(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                 void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream) {
+    if (!features || !out_tokens || !out_count || !out_pos_thw) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    Scratch s;
+    carve_scratch(p, nullptr, &s);
+    void* ws = nullptr;
+    rc = cached_scratch(s.bytes, (cudaStream_t)stream, &ws);
+    if (rc != TTF_OK) return rc;
+    return compress_impl(p, ws, out_tokens, out_count, out_pos_thw, (cudaStream_t)stream);
+}
+
+int ttf_query_ws(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                 int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
+                 int* out_fuse_cnt, void* workspace, size_t workspace_bytes, ttf_stream_t stream) {
+    if (!features) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    Scratch s;
+    rc = check_ws(p, workspace, workspace_bytes, &s);
+    if (rc != TTF_OK) return rc;
+    return query_impl(p, workspace, out_anchor, out_keep, out_dst, out_best_sim, out_fuse_cnt,
+                      (cudaStream_t)stream);
+}
+
+int ttf_query(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+              int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
+              int* out_fuse_cnt, ttf_stream_t stream) {
+    if (!features) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    Scratch s;
+    carve_scratch(p, nullptr, &s);
+    void* ws = nullptr;
+    rc = cached_scratch(s.bytes, (cudaStream_t)stream, &ws);
+    if (rc != TTF_OK) return rc;
+    return query_impl(p, ws, out_anchor, out_keep, out_dst, out_best_sim, out_fuse_cnt, (cudaStream_t)stream);
+}
+
+int ttf_compress_host(const void* features_host, int F, int H, int W, int C, int r, float t, int dtype,
+                      void* out_tokens_host, int* out_count_host, int* out_pos_thw_host) {
+    if (!features_host || !out_tokens_host || !out_count_host || !out_pos_thw_host) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    // the staging copy is always 256-byte aligned: validate with an aligned stand-in pointer
+    int rc = make_problem(reinterpret_cast<const void*>(uintptr_t(256)), F, H, W, C, r, t, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const size_t esize = dtype == TTF_DTYPE_F32 ? 4 : 2;
+    const size_t FN = (size_t)p.F * p.N;
+    const size_t row_bytes = (size_t)C * esize;
+
+    std::unique_lock<std::mutex> lk(g_mu);
+    Staging& sg = g_staging[dev];
+    if (!sg.stream) {
+        e = cudaStreamCreateWithFlags(&sg.stream, cudaStreamNonBlocking);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (!sg.count) {
+        e = cudaMalloc((void**)&sg.count, 256);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    e = grow(&sg.feat, &sg.feat_bytes, FN * row_bytes);
+    if (e == cudaSuccess) e = grow(&sg.tok, &sg.tok_bytes, FN * row_bytes);
+    if (e == cudaSuccess) e = grow((void**)&sg.pos, &sg.pos_bytes, FN * 3 * sizeof(int));
+    if (e != cudaSuccess) return cuda_fail(e);
+    Staging local = sg;
+    lk.unlock();
+
+    cudaStream_t st = local.stream;
+    e = cudaMemcpyAsync(local.feat, features_host, FN * row_bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    rc = ttf_compress(local.feat, F, H, W, C, r, t, dtype, local.tok, local.count, local.pos, st);
+    if (rc != TTF_OK) return rc;
+    e = cudaMemcpyAsync(out_count_host, local.count, sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const size_t L = (size_t)*out_count_host;
+    if (L > FN) return TTF_ERR_CUDA;
+    e = cudaMemcpyAsync(out_tokens_host, local.tok, L * row_bytes, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_pos_thw_host, local.pos, L * 3 * sizeof(int), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return TTF_OK;
+}
+
+int ttf_release(void) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    int cur = 0;
+    cudaGetDevice(&cur);
+    cudaError_t first = cudaSuccess;
+    for (auto& kv : g_scratch) {
+        cudaSetDevice(kv.first.first);
+        cudaError_t e = cudaDeviceSynchronize();
+        if (e != cudaSuccess && first == cudaSuccess) first = e;
+        if (kv.second.ptr) cudaFree(kv.second.ptr);
+    }
+    g_scratch.clear();
+    for (auto& kv : g_staging) {
+        cudaSetDevice(kv.first);
+        cudaError_t e = cudaDeviceSynchronize();
+        if (e != cudaSuccess && first == cudaSuccess) first = e;
+        Staging& s = kv.second;
+        if (s.feat) cudaFree(s.feat);
+        if (s.tok) cudaFree(s.tok);
+        if (s.pos) cudaFree(s.pos);
+        if (s.count) cudaFree(s.count);
+        if (s.stream) cudaStreamDestroy(s.stream);
+    }
+    g_staging.clear();
+    cudaSetDevice(cur);
+    return first == cudaSuccess ? TTF_OK : cuda_fail(first);
+}
+
+}  // extern "C"

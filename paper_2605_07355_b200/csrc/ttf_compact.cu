@@ -1,0 +1,217 @@
+// Token Compression and Positional Alignment (Eqs. xprime_stack, mask, compress_pos, Lpre), plus the
+// bookkeeping of identity replacement (how many source tokens each anchor cell absorbed).
+//
+// The output position of a preserved source token is N plus the number of preserved source tokens before it
+// in flat (k, i) order.  That exclusive prefix is taken in two levels: the per-frame survivor counts written
+// by the matching kernel are scanned by every CTA (shared memory, or a pre-scanned array for very long
+// clips), and inside a frame the rank is a population count over the frame's keep flags.  The gather is then
+// driven from the OUTPUT side: work item (output row j, 2 KB part of the row) -> rank/select finds the source
+// row, so every warp copies the same number of bytes no matter how unevenly the survivors are spread over
+// the frames.  No CTA ever waits for another one.
+#include "ttf_internal.cuh"
+
+namespace ttf {
+
+constexpr int kCopyWarps = 8;
+constexpr int kPartBytes = 2048;     // bytes of one row handled by one warp-level work item
+
+// exclusive scan of the effective per-frame counts (anchor frame counts as 0) for clips with more frames
+// than fit the shared-memory scan of the gather kernel
+__global__ void __launch_bounds__(1024)
+k_frame_prefix(const int* __restrict__ cnt, const int* __restrict__ hdr, int F, int* __restrict__ prefix)
+{
+    __shared__ int s_warp[32];
+    __shared__ int s_carry;
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int a = hdr[HDR_ANCHOR];
+    if (tid == 0) s_carry = 0;
+    __syncthreads();
+    for (int base = 0; base < F; base += 1024) {
+        const int k = base + tid;
+        int v = (k < F && k != a) ? cnt[k] : 0;
+        int incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int n = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += n;
+        }
+        if (lane == 31) s_warp[w] = incl;
+        __syncthreads();
+        if (w == 0) {
+            int x = s_warp[lane], xi = x;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int n = __shfl_up_sync(0xffffffffu, xi, o);
+                if (lane >= o) xi += n;
+            }
+            s_warp[lane] = xi - x;       // exclusive over warps
+        }
+        __syncthreads();
+        const int carry = s_carry;
+        if (k < F) prefix[k] = carry + s_warp[w] + incl - v;
+        __syncthreads();
+        if (tid == 1023) s_carry = carry + s_warp[w] + incl;
+        __syncthreads();
+    }
+    if (tid == 0) prefix[F] = s_carry;
+}
+
+// COPY_BYTES: 16 when rows are 16-byte aligned multiples of 16 bytes, else the element size (2 or 4)
+template <int COPY_BYTES> struct CopyUnit;
+template <> struct CopyUnit<16> { using type = uint4; };
+template <> struct CopyUnit<4> { using type = uint32_t; };
+template <> struct CopyUnit<2> { using type = uint16_t; };
+
+template <int COPY_BYTES>
+__global__ void __launch_bounds__(kCopyWarps * 32)
+k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, int W, int r,
+          const int* __restrict__ hdr, const int* __restrict__ cnt, const int* __restrict__ gprefix,
+          const unsigned char* __restrict__ keep, const int* __restrict__ dst,
+          unsigned char* __restrict__ out_tokens, int* __restrict__ out_pos, int* __restrict__ out_count,
+          int* __restrict__ fuse_cnt, int ncopy_blocks, int parts_per_row)
+{
+    using U = typename CopyUnit<COPY_BYTES>::type;
+    const int N = H * W;
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int a = hdr[HDR_ANCHOR];
+
+    // ---- bookkeeping CTAs: tokens fused into each anchor cell (gather-side, integer, fixed order) --------
+    if ((int)blockIdx.x >= ncopy_blocks) {
+        if (fuse_cnt == nullptr) return;
+        const int nb = gridDim.x - ncopy_blocks;
+        for (int j = ((int)blockIdx.x - ncopy_blocks) * kCopyWarps + w; j < N; j += nb * kCopyWarps) {
+            const int y = j / W, x = j - y * W;
+            int c = 0;
+            for (int k = lane; k < F; k += 32) {
+                if (k == a) continue;
+                for (int yy = max(0, y - r); yy <= min(H - 1, y + r); ++yy)
+                    for (int xx = max(0, x - r); xx <= min(W - 1, x + r); ++xx) {
+                        const size_t f = (size_t)k * N + yy * W + xx;
+                        c += (!keep[f] && dst[f] == j) ? 1 : 0;
+                    }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+            if (lane == 0) fuse_cnt[j] = c;
+        }
+        return;
+    }
+
+    // ---- exclusive prefix of preserved tokens per frame ------------------------------------------------
+    __shared__ int s_pre[kSmemPrefixMaxF + 1];
+    __shared__ int s_warp[kCopyWarps];
+    const int* pre;
+    if (F <= kSmemPrefixMaxF) {
+        // each thread scans a contiguous run of frames, runs are combined over the block in thread order
+        const int per = (F + kCopyWarps * 32 - 1) / (kCopyWarps * 32);
+        const int k0 = tid * per;
+        int sum = 0;
+        for (int k = k0; k < min(F, k0 + per); ++k) sum += (k != a) ? cnt[k] : 0;
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int n = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += n;
+        }
+        if (lane == 31) s_warp[w] = incl;
+        __syncthreads();
+        int woff = 0;
+        for (int ww = 0; ww < w; ++ww) woff += s_warp[ww];
+        int run = woff + incl - sum;
+        for (int k = k0; k < min(F, k0 + per); ++k) { s_pre[k] = run; run += (k != a) ? cnt[k] : 0; }
+        if (tid == kCopyWarps * 32 - 1) s_pre[F] = woff + incl;
+        __syncthreads();
+        pre = s_pre;
+    } else {
+        pre = gprefix;
+    }
+    const int P = pre[F];
+    const int L = N + P;                                   // L' = N + P (Eq. Lpre)
+    if (blockIdx.x == 0 && tid == 0) { *out_count = L; }
+
+    // ---- output-driven gather ---------------------------------------------------------------------------
+    const long long items = (long long)L * parts_per_row;
+    const long long stride = (long long)ncopy_blocks * kCopyWarps;
+    const int units_per_row = (int)(row_bytes / COPY_BYTES);
+    const int units_per_part = kPartBytes / COPY_BYTES;
+    for (long long it = (long long)blockIdx.x * kCopyWarps + w; it < items; it += stride) {
+        const int j = (int)(it / parts_per_row);
+        const int part = (int)(it - (long long)j * parts_per_row);
+        int k, i;
+        if (j < N) { k = a; i = j; }                        // anchor rows first (Eq. xprime_stack)
+        else {
+            const int e = j - N;
+            int lo = 0, hi = F;                             // largest k with pre[k] <= e
+            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (pre[mid] <= e) lo = mid; else hi = mid; }
+            k = lo;
+            int n = e - pre[k];                             // rank inside frame k
+            const unsigned char* kf = keep + (size_t)k * N;
+            i = -1;
+            for (int b = 0; b < N; b += 32) {
+                const int ii = b + lane;
+                const unsigned m = __ballot_sync(0xffffffffu, ii < N && kf[ii] != 0);
+                const int c = __popc(m);
+                if (n < c) { i = b + (int)__fns(m, 0, n + 1); break; }
+                n -= c;
+            }
+            if (i < 0) continue;                            // cannot happen when cnt matches keep
+        }
+        const size_t f = (size_t)k * N + i;
+        const U* src = reinterpret_cast<const U*>(X + f * row_bytes);
+        U* dsto = reinterpret_cast<U*>(out_tokens + (size_t)j * row_bytes);
+        const int u0 = part * units_per_part;
+        const int u1 = min(units_per_row, u0 + units_per_part);
+        for (int u = u0 + lane; u < u1; u += 32 * 4) {
+            U v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) if (u + q * 32 < u1) v[q] = src[u + q * 32];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) if (u + q * 32 < u1) dsto[u + q * 32] = v[q];
+        }
+        if (part == 0 && lane < 3) {                        // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
+            const int yy = i / W;
+            out_pos[(size_t)j * 3 + lane] = lane == 0 ? k : (lane == 1 ? yy : i - yy * W);
+        }
+    }
+}
+
+cudaError_t launch_fuse_count(const Problem& p, const Scratch& s, const int* dst, const unsigned char* keep,
+                              int* fuse_cnt, cudaStream_t st) {
+    // bookkeeping only: the same kernel with zero copy CTAs
+    const int nb = (p.N + kCopyWarps - 1) / kCopyWarps;
+    k_compact<4><<<nb < 1024 ? nb : 1024, kCopyWarps * 32, 0, st>>>(
+        nullptr, 0, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix, keep, dst, nullptr, nullptr, nullptr,
+        fuse_cnt, 0, 1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens, int* out_pos, int* out_count,
+                           cudaStream_t st) {
+    const size_t esize = p.dtype == 0 ? 4 : 2;
+    const size_t row_bytes = (size_t)p.C * esize;
+    const bool vec = p.vec && (reinterpret_cast<uintptr_t>(out_tokens) % 16 == 0);
+    if (p.F > kSmemPrefixMaxF) {
+        k_frame_prefix<<<1, 1024, 0, st>>>(s.cnt, s.hdr, p.F, s.prefix);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    const int parts = (int)((row_bytes + kPartBytes - 1) / kPartBytes);
+    const int ncopy = 2 * sm_count();
+    int nfuse = (p.N + kCopyWarps - 1) / kCopyWarps;
+    if (nfuse > sm_count()) nfuse = sm_count();
+    const int grid = ncopy + nfuse;
+    const unsigned char* X = reinterpret_cast<const unsigned char*>(p.X);
+    unsigned char* out = reinterpret_cast<unsigned char*>(out_tokens);
+    if (vec)
+        k_compact<16><<<grid, kCopyWarps * 32, 0, st>>>(X, row_bytes, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix,
+            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy, parts);
+    else if (esize == 4)
+        k_compact<4><<<grid, kCopyWarps * 32, 0, st>>>(X, row_bytes, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix,
+            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy, parts);
+    else
+        k_compact<2><<<grid, kCopyWarps * 32, 0, st>>>(X, row_bytes, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix,
+            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy, parts);
+    return cudaGetLastError();
+}
+
+}  // namespace ttf

@@ -1,0 +1,112 @@
+// Shared declarations of the TTF kernels: scratch layout, launch entry points, small device helpers.
+// Paper references are to arXiv 2605.07355, Sec. 3.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+namespace ttf {
+
+constexpr float kNormFloor = 1e-12f;   // norms are floored here before dividing (zero token -> similarity 0)
+constexpr int kSmemPrefixMaxF = 2048;  // frame counts up to this are scanned in shared memory by the gather
+constexpr int kHdrInts = 64;
+
+// header words of the scratch block
+enum { HDR_ANCHOR = 0, HDR_COUNT = 1, HDR_DONE0 = 2, HDR_DONE1 = 3 };
+
+// Problem description handed to every launcher.
+struct Problem {
+    const void* X;      // [F, N, C]
+    int F, H, W, C, r;
+    float t;
+    int dtype;          // 0 fp32, 1 bf16
+    int N;              // H * W
+    int vec;            // 1 when rows are 16-byte aligned and a multiple of 16 bytes long, else 0
+    int lanes_elems;    // channels one lane loads at once: 16 B worth when vec, else 1
+    int nslice;         // channel slices of 32 lanes: ceil(C / (32 * lanes_elems))
+    int anchor_mode;    // 0 auto (Eq. auto_anchor), 1 first, 2 last, 3 explicit
+    int anchor_arg;     // explicit anchor frame
+};
+
+// Device pointers carved out of one scratch allocation.
+struct Scratch {
+    int* hdr;           // [kHdrInts]
+    int* cnt;           // [F]   preserved tokens per source frame (Eq. gating summed over a frame)
+    int* prefix;        // [F+1] exclusive scan of cnt, only used when F > kSmemPrefixMaxF
+    float* fcos;        // [F]   cosine of each frame mean to the global mean (Eq. auto_anchor)
+    float* g;           // [C]   sum of all tokens
+    float* S;           // [F, C] per-frame channel sums
+    float* ssq;         // [nslice, F*N] partial squared norms per channel slice
+    float* shat;        // [F*N] best similarity (Eq. argmax)
+    int* dst;           // [F*N] best anchor cell (Eq. dst)
+    unsigned char* keep;// [F*N] retention mask (Eq. mask)
+    int* fuse_cnt;      // [N]   tokens fused into each anchor cell
+    size_t bytes;       // total, multiple of 256
+};
+
+// Fills the offsets (base may be NULL to only compute `bytes`).
+void carve_scratch(const Problem& p, void* base, Scratch* s);
+
+// Kernel launchers (each enqueues on `st` and returns the launch error, if any).
+cudaError_t launch_norm_sum(const Problem& p, const Scratch& s, cudaStream_t st);
+cudaError_t launch_anchor_pick(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st);
+cudaError_t launch_match(const Problem& p, const Scratch& s, float* shat, int* dst, unsigned char* keep,
+                         cudaStream_t st);
+cudaError_t launch_fuse_count(const Problem& p, const Scratch& s, const int* dst, const unsigned char* keep,
+                              int* fuse_cnt, cudaStream_t st);
+cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens, int* out_pos, int* out_count,
+                           cudaStream_t st);
+
+int sm_count();   // SMs of the current device (cached per device)
+
+// ---------------------------------------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+struct bf16_t { uint16_t bits; };   // storage type only: all arithmetic is on the widened fp32 value
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// Loads V consecutive channels starting at p (p is 16-byte aligned when V > 1) and widens them to fp32.
+template <typename T, int V> struct Loader;
+template <> struct Loader<float, 4> {
+    static __device__ __forceinline__ void load(const float* p, float (&x)[4]) {
+        float4 v = __ldg(reinterpret_cast<const float4*>(p));
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    }
+};
+template <> struct Loader<float, 1> {
+    static __device__ __forceinline__ void load(const float* p, float (&x)[1]) { x[0] = __ldg(p); }
+};
+template <> struct Loader<bf16_t, 8> {
+    static __device__ __forceinline__ void load(const bf16_t* p, float (&x)[8]) {
+        uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+        x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);
+        x[4] = bf16_lo(v.z); x[5] = bf16_hi(v.z); x[6] = bf16_lo(v.w); x[7] = bf16_hi(v.w);
+    }
+};
+template <> struct Loader<bf16_t, 1> {
+    static __device__ __forceinline__ void load(const bf16_t* p, float (&x)[1]) {
+        x[0] = __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
+    }
+};
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// 1 / max(||x||, floor) from the per-slice partial squared norms of token f, summed in slice order
+__device__ __forceinline__ float inv_norm(const float* __restrict__ ssq, int nslice, size_t FN, size_t f) {
+    float s = 0.f;
+    for (int q = 0; q < nslice; ++q) s += ssq[(size_t)q * FN + f];
+    return 1.0f / fmaxf(sqrtf(s), kNormFloor);
+}
+
+#endif  // __CUDACC__
+
+}  // namespace ttf

@@ -1,0 +1,70 @@
+"""Host-side checks that need no GPU: the C-ABI library loads, exports every symbol include/ttf.h declares,
+and rejects invalid arguments before any CUDA call."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2605_07355_b200 as P
+from paper_2605_07355_b200 import build as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    B.build()
+    return P.lib()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "ttf.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"^\s*(?:const\s+char\s*\*|int)\s+(ttf_\w+)\s*\(", text, flags=re.M)
+    return sorted(set(names))
+
+
+def test_header_symbols_are_exported(lib):
+    names = declared_symbols()
+    assert "ttf_compress" in names and "ttf_query" in names and len(names) >= 9
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(names) == set(P.EXPORTS)
+
+
+def test_status_strings(lib):
+    assert lib.ttf_status_string(0) == b"TTF_OK"
+    assert lib.ttf_status_string(1) == b"TTF_ERR_INVALID_ARG"
+    assert lib.ttf_status_string(99) == b"TTF_ERR_UNKNOWN"
+
+
+def test_workspace_bytes_and_validation(lib):
+    n = P.ttf_workspace_bytes(32, 16, 16, 4096, 1, P.TTF_DTYPE_BF16)
+    assert n % 256 == 0 and n > 32 * 4096 * 4
+    assert P.ttf_workspace_bytes(64, 32, 32, 4096, 2, P.TTF_DTYPE_BF16) > n
+    sz = ctypes.c_size_t(0)
+    bad = [(0, 4, 4, 8, 1, 0), (4, 0, 4, 8, 1, 0), (4, 4, 4, 0, 1, 0), (4, 4, 4, 8, -1, 0), (4, 4, 4, 8, 1, 7)]
+    for args in bad:
+        assert lib.ttf_workspace_bytes(*args, ctypes.byref(sz)) == 1
+    assert lib.ttf_workspace_bytes(1 << 16, 1 << 8, 1 << 8, 8, 1, 0, ctypes.byref(sz)) == 2     # F*H*W >= 2^31
+    assert lib.ttf_workspace_bytes(4, 4, 4, 8, 1, 0, None) == 1
+
+
+def test_null_and_nonfinite_arguments_are_rejected_before_any_launch(lib):
+    fake = ctypes.c_void_p(4096)        # never dereferenced: validation fails first
+    f = lib.ttf_compress
+    assert f(None, 4, 4, 4, 8, 1, 0.7, 0, fake, fake, fake, None) == 1
+    assert f(fake, 4, 4, 4, 8, 1, 0.7, 0, None, fake, fake, None) == 1
+    assert f(fake, 4, 4, 4, 8, 1, float("nan"), 0, fake, fake, fake, None) == 1
+    assert f(fake, 4, 4, 4, 8, 1, float("inf"), 0, fake, fake, fake, None) == 1
+    assert f(fake, 4, 4, 4, 8, -1, 0.7, 0, fake, fake, fake, None) == 1
+    assert f(fake, 4, 4, 4, 8, 1, 0.7, 3, fake, fake, fake, None) == 1
+    assert lib.ttf_compress_ws(fake, 4, 4, 4, 8, 1, 0.7, 0, fake, fake, fake, None, 0, None) == 3
+    assert lib.ttf_compress_ws(fake, 4, 4, 4, 8, 1, 0.7, 0, fake, fake, fake, ctypes.c_void_p(4096 + 8), 1 << 30, None) == 3
+    assert lib.ttf_query(None, 4, 4, 4, 8, 1, 0.7, 0, None, None, None, None, None, None) == 1
+    assert lib.ttf_compress_host(None, 4, 4, 4, 8, 1, 0.7, 0, fake, fake, fake) == 1
+
+
+def test_decode_alignment_helper():
+    assert P.ttf_decode_pos(2703, 57, 0) == 2760 and P.ttf_decode_pos(2703, 57, 4) == 2764
