@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Throughput of the TTF pass on B200: visual tokens/s and clips/s through ttf_compress, roofline fraction of
+the dominant kernel, end-to-end rate through the host-buffer entry point, and the CPU oracle timed beside it.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload NAME] [--clips B] [--streams S] [--no-e2e] [--no-cpu]
+
+A step is one pass of the whole path (norm/frame-sum sweep, anchor pick, windowed match + gate, compaction
+with positions and fuse bookkeeping) over a batch of B distinct synthetic clips of the workload, one
+ttf_compress call per clip.  The batch is larger than L2, so every clip starts cold in HBM.  Rank 0 prints
+one JSON line.  With N > 1 (torchrun) every rank runs the same batch shape on its own GPU: clips are
+independent, there is no collective on the data path (weak scaling, replicas).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "visual tokens/s through TTF"
+UNIT = "tokens/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="vl8b_cal")
+    ap.add_argument("--clips", type=int, default=16, help="distinct clips per step (batch)")
+    ap.add_argument("--streams", type=int, default=1, help="CUDA streams the clips of a step are spread over")
+    ap.add_argument("--threshold", type=float, default=None)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    return ap.parse_args()
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            d = json.load(open(path))
+            return float(d["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+# ---------------------------------------------------------------------------------------------------------
+# clock sampling (reads only; never changes a GPU setting)
+# ---------------------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, torch_device: int, period_s: float = 0.02):
+        self.samples = []           # (time, sm_mhz, reasons bitmask)
+        self.period = period_s
+        self.handle = None
+        self.max_mhz = None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(torch_device).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            try:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            self.nv = pynvml
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM))
+        except Exception as e:      # no NVML: the JSON says so
+            self.error = repr(e)
+
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+                try:
+                    rs = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle))
+                except Exception:
+                    rs = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle))
+                self.samples.append((time.perf_counter(), mhz, rs))
+            except Exception:
+                pass
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self.handle is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self, t0: float, t1: float) -> dict:
+        if self.handle is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "note": "NVML unavailable"}
+        window = "timed"
+        sel = [s for s in self.samples if t0 <= s[0] <= t1]
+        if len(sel) < 3:
+            sel, window = self.samples, "run"
+        if not sel:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "note": "no samples"}
+        bits = 0
+        for _, _, rs in sel:
+            bits |= rs
+        reasons = sorted(name for bit, name in self.REASONS.items() if bits & bit)
+        return {"sm_mhz": statistics.median(s[1] for s in sel), "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(sel), "window": window}
+
+
+# ---------------------------------------------------------------------------------------------------------
+# reference arm / CPU baseline: the oracle as it stands, on the host cores
+# ---------------------------------------------------------------------------------------------------------
+def oracle_sample_plan(spec, t, budget_s_per_step):
+    """Times the oracle on one clip, then sizes a step's sample to the budget."""
+    from oracle import ttf_oracle as O
+    from paper_2605_07355_b200 import clips
+    X = clips.make_clip(spec, spec.seed)
+    t0 = time.perf_counter()
+    O.compress(X, spec.r, t)
+    one = time.perf_counter() - t0
+    if one <= budget_s_per_step:
+        n = max(1, min(4, int(budget_s_per_step / one)))
+        Xs = [X] + [clips.make_clip(spec, spec.seed + j) for j in range(1, n)]
+        desc = f"{n} whole clip(s) of {spec.name} per step"
+    else:
+        frames = max(2, int(spec.F * budget_s_per_step / one))
+        Xs = [np.ascontiguousarray(X[:frames])]
+        desc = f"first {frames} of {spec.F} frames of one {spec.name} clip per step"
+    return Xs, desc
+
+
+def run_oracle_steps(Xs, spec, t, steps, warmup):
+    from oracle import ttf_oracle as O
+    tokens = sum(x.shape[0] * x.shape[1] * x.shape[2] for x in Xs)
+    for _ in range(warmup):
+        for x in Xs:
+            O.compress(x, spec.r, t)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        for x in Xs:
+            O.compress(x, spec.r, t)
+    dt = time.perf_counter() - t0
+    return tokens * steps / dt, dt / steps * 1e3, tokens
+
+
+def reference_arm(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import ttf_oracle as O
+    from paper_2605_07355_b200 import clips
+    spec = clips.CONFIGS[args.workload]
+    t = spec.t if args.threshold is None else args.threshold
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    Xs, desc = oracle_sample_plan(spec, t, budget)
+    value, ms, tokens = run_oracle_steps(Xs, spec, t, args.steps, args.warmup)
+    cores = O.threads()
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(spec, t, len(Xs), 0, tokens),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(spec, t, clips_per_step, streams, tokens_per_step):
+    return {"workload": f"{spec.name}: F={spec.F} {spec.H}x{spec.W} C={spec.C} {spec.dtype} r={spec.r} t={t:.2f}",
+            "generator": spec.family, "clips_per_step": clips_per_step, "tokens_per_step": tokens_per_step,
+            "streams": streams,
+            "l2": "inputs rotate through a batch larger than L2; every clip starts cold in HBM"}
+
+
+# ---------------------------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        reference_arm(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2605_07355_b200 import build as B
+    from paper_2605_07355_b200 import accounting as A
+    from paper_2605_07355_b200 import clips
+    import paper_2605_07355_b200 as P
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if rank == 0:
+        B.build()
+    if world > 1:
+        dist.barrier()
+    P.lib()
+
+    spec = clips.CONFIGS[args.workload]
+    t = spec.t if args.threshold is None else args.threshold
+    nclips = args.clips
+    FN, C = spec.tokens, spec.C
+    clip_bytes = FN * C * spec.itemsize
+    tdtype = torch.float32 if spec.dtype == "f32" else torch.bfloat16
+
+    # ---- inputs: pinned host copies (for the end-to-end leg) and device-resident copies -------------------
+    host, devX = [], []
+    for j in range(nclips):
+        Xn = clips.make_clip(spec, spec.seed + 1000 * rank + j)
+        th = torch.from_numpy(Xn if spec.dtype == "f32" else Xn.view(np.int16))
+        th = (th if spec.dtype == "f32" else th.view(torch.bfloat16)).pin_memory()
+        host.append(th)
+        devX.append(th.to(dev, non_blocking=True))
+    out_tok = [torch.empty((FN, C), dtype=tdtype, device=dev) for _ in range(nclips)]
+    out_cnt = [torch.empty(1, dtype=torch.int32, device=dev) for _ in range(nclips)]
+    out_pos = [torch.empty((FN, 3), dtype=torch.int32, device=dev) for _ in range(nclips)]
+    torch.cuda.synchronize()
+
+    nstreams = max(1, args.streams)
+    main_stream = torch.cuda.Stream(device=dev)
+    streams = [main_stream] if nstreams == 1 else [torch.cuda.Stream(device=dev) for _ in range(nstreams)]
+    fork = torch.cuda.Event()
+    joins = [torch.cuda.Event() for _ in streams]
+
+    def step():
+        if nstreams == 1:
+            for j in range(nclips):
+                P.ttf_compress(devX[j], spec.r, t, out_tok[j], out_cnt[j], out_pos[j], stream=main_stream)
+            return
+        fork.record(main_stream)
+        for s in streams:
+            s.wait_event(fork)
+        for j in range(nclips):
+            P.ttf_compress(devX[j], spec.r, t, out_tok[j], out_cnt[j], out_pos[j], stream=streams[j % nstreams])
+        for s, ev in zip(streams, joins):
+            ev.record(s)
+            main_stream.wait_event(ev)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    barrier()
+    counts = [int(c.item()) for c in out_cnt]
+    rho = 1.0 - sum(counts) / float(nclips * FN)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.05)
+
+    # ---- timed region: exactly K steps, CUDA events on the launching stream -------------------------------
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    w0 = time.perf_counter()
+    e0.record(main_stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(main_stream)
+    barrier()
+    w1 = time.perf_counter()
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        tmax = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms_total = float(tmax.item())
+    ms_step = ms_total / args.steps
+    tokens_step = nclips * FN
+    value = world * tokens_step / (ms_step * 1e-3)
+    clips_per_s = world * nclips / (ms_step * 1e-3)
+
+    # ---- per-kernel durations: the same steps again with events around every launch -----------------------
+    prof_steps = min(args.steps, 50)
+    P.ttf_profile_begin()
+    for _ in range(prof_steps):
+        step()
+    torch.cuda.synchronize()
+    prof = P.ttf_profile_end()
+    sampler.stop()
+    clocks = sampler.summary(w0, w1)
+
+    launches_per_step = sum(v[1] for v in prof.values()) // prof_steps
+    kern = {k: {"launches": v[1], "us_per_launch": 1e3 * v[0] / v[1]} for k, v in prof.items() if v[1]}
+    tot = sum(v[0] for v in prof.values())
+    dominant = max(kern, key=lambda k: prof[k][0])
+    peak_gbs, peak_kind = peaks()
+    avg_count = sum(counts) / nclips
+    nslice = (C + 32 * (16 // spec.itemsize) - 1) // (32 * (16 // spec.itemsize))
+    kbytes = A.kernel_bytes(dominant, spec.F, spec.N, C, spec.itemsize, int(round(avg_count)), nslice)
+    achieved = kbytes / (kern[dominant]["us_per_launch"] * 1e-6) / 1e9
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
+                "frac": achieved / peak_gbs, "peak_source": f"of {peak_kind}", "traffic": None,
+                "algorithmic_bytes_per_launch": kbytes,
+                "kernel_share": {k: prof[k][0] / tot for k in kern},
+                "kernel_us": {k: round(kern[k]["us_per_launch"], 3) for k in kern}}
+    bmin = A.pass_bytes(spec.F, spec.N, C, spec.itemsize, int(round(avg_count)))
+    pass_gbs = bmin * nclips / (ms_step * 1e-3) / 1e9
+    pass_roofline = {"bytes_per_clip": bmin, "achieved": pass_gbs, "unit": "GB/s", "frac_of_measured_copy": pass_gbs / peak_gbs,
+                     "frac_of_8TBps": pass_gbs / 8000.0, "us_per_clip": ms_step * 1e3 / nclips}
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region --------------------
+    e2e = None
+    if not args.no_e2e:
+        h_tok = torch.empty((FN, C), dtype=tdtype).pin_memory()
+        h_pos = torch.empty((FN, 3), dtype=torch.int32).pin_memory()
+        for j in range(min(2, nclips)):
+            P.ttf_compress_host(host[j], spec.r, t, h_tok, h_pos)
+        barrier()
+        d2h = 0
+        t0 = time.perf_counter()
+        for _ in range(args.e2e_steps):
+            d2h = 0
+            for j in range(nclips):
+                _, L, _ = P.ttf_compress_host(host[j], spec.r, t, h_tok, h_pos)
+                d2h += L * (C * spec.itemsize + 12) + 4
+        barrier()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            tm = torch.tensor([dt], dtype=torch.float64, device=dev)
+            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+            dt = float(tm.item())
+        e2e = {"value": world * tokens_step * args.e2e_steps / dt, "unit": UNIT,
+               "h2d_bytes_per_step": nclips * clip_bytes, "d2h_bytes_per_step": d2h,
+               "steps": args.e2e_steps, "api": "ttf_compress_host (pinned host buffers)"}
+
+    # ---- the oracle on the host cores (rank 0, N = 1 only) ------------------------------------------------
+    cpu = None
+    if not args.no_cpu and world == 1 and rank == 0:
+        from oracle import ttf_oracle as O
+        Xs, desc = oracle_sample_plan(spec, t, args.cpu_seconds / 3.0)
+        v, _, _ = run_oracle_steps(Xs, spec, t, 3, 0)
+        cpu = {"value": v, "unit": UNIT, "cores": O.threads(), "kind": "oracle", "sample": desc + ", 3 steps"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": workload_config(spec, t, nclips, nstreams, tokens_step),
+            "clips_per_s": clips_per_s, "rho": rho, "count_mean": avg_count,
+            "roofline": roofline, "pass_roofline": pass_roofline, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": int(launches_per_step * args.steps), "gpu_launches_per_step": int(launches_per_step),
+            "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,42 @@
+"""Algorithmic bytes and flops of the TTF pass (host arithmetic only; used by the benchmark's roofline).
+
+"Algorithmic" = what the method must move or compute for one clip, independent of how kernels are organised:
+the pass has to read X once and write X', P' and L' (Eqs. xprime_stack, compress_pos, Lpre).
+"""
+from __future__ import annotations
+
+
+def window_pairs(H: int, W: int, r: int) -> int:
+    """sum over cells of |J(i)|: candidates left by clipping (Eq. pi) and duplicate masking."""
+    ny = sum(min(H - 1, y + r) - max(0, y - r) + 1 for y in range(H))
+    nx = sum(min(W - 1, x + r) - max(0, x - r) + 1 for x in range(W))
+    return ny * nx
+
+
+def matching_flops_nominal(F: int, N: int, C: int, r: int) -> int:
+    """The paper's count of the matching overhead: 2 (F-1) N (2r+1)^2 C (cost term O((2r+1)^2 FNC); Table 3)."""
+    return 2 * (F - 1) * N * (2 * r + 1) ** 2 * C
+
+
+def matching_flops(F: int, H: int, W: int, C: int, r: int) -> int:
+    """Multiply-adds actually needed (border cells have fewer candidates), as flops."""
+    return 2 * (F - 1) * window_pairs(H, W, r) * C
+
+
+def pass_bytes(F: int, N: int, C: int, itemsize: int, count: int) -> int:
+    """B_min: read X once; write X' (count rows), P' (count x 3 int32) and L'."""
+    return F * N * C * itemsize + count * C * itemsize + count * 12 + 4
+
+
+def kernel_bytes(kind: str, F: int, N: int, C: int, itemsize: int, count: int, nslice: int) -> int:
+    """Algorithmic bytes of one launch of each kernel kind."""
+    X = F * N * C * itemsize
+    if kind == "norm_sum":          # reads X; writes frame sums and per-slice squared norms
+        return X + F * C * 4 + nslice * F * N * 4
+    if kind == "match":             # reads X (sources + anchor frame once); writes s_hat, dst, keep
+        return X + F * N * 9
+    if kind == "compact":           # reads the retained rows, writes them with their positions
+        return 2 * count * C * itemsize + count * 12 + F * N + 4
+    if kind == "anchor_pick":
+        return 2 * F * C * 4
+    raise KeyError(kind)

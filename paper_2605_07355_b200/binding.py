@@ -20,8 +20,9 @@ TTF_OK = 0
 
 EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
-    "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release",
+    "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
 ]
+KERNEL_KINDS = ["norm_sum", "anchor_pick", "match", "compact", "frame_prefix", "fuse_count"]
 
 _lib = None
 
@@ -62,6 +63,10 @@ def lib() -> ctypes.CDLL:
         L.ttf_compress_host.argtypes = [vp] + shape + [f, i, vp, vp, vp]
         L.ttf_release.restype = i
         L.ttf_release.argtypes = []
+        L.ttf_profile_begin.restype = i
+        L.ttf_profile_begin.argtypes = []
+        L.ttf_profile_end.restype = i
+        L.ttf_profile_end.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_longlong), i]
         _lib = L
     return _lib
 
@@ -182,6 +187,23 @@ def ttf_release() -> None:
     rc = lib().ttf_release()
     if rc != TTF_OK:
         raise TTFError(rc, "ttf_release")
+
+
+def ttf_profile_begin() -> None:
+    rc = lib().ttf_profile_begin()
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_profile_begin")
+
+
+def ttf_profile_end() -> dict:
+    """Returns {kernel kind: (total device ms, launches)} for the launches since ttf_profile_begin."""
+    n = len(KERNEL_KINDS)
+    ms = (ctypes.c_double * n)()
+    cnt = (ctypes.c_longlong * n)()
+    rc = lib().ttf_profile_end(ms, cnt, n)
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_profile_end")
+    return {k: (float(ms[i]), int(cnt[i])) for i, k in enumerate(KERNEL_KINDS)}
 
 
 def ttf_decode_pos(L_prime: int, T: int, l: int) -> int:

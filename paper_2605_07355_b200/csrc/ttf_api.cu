@@ -32,6 +32,29 @@ int sm_count() {
     return n;
 }
 
+// ---- optional per-kernel timing: CUDA events recorded around every launch while profiling is on ---------
+enum { PK_NORM_SUM = 0, PK_ANCHOR_PICK = 1, PK_MATCH = 2, PK_COMPACT = 3, PK_FRAME_PREFIX = 4, PK_FUSE_COUNT = 5,
+       PK_KINDS = 6 };
+struct ProfRecord { int kind; cudaEvent_t a, b; };
+static std::mutex g_prof_mu;
+static bool g_prof_on = false;
+static std::vector<ProfRecord> g_prof;
+
+struct ProfScope {
+    cudaStream_t st; int kind; cudaEvent_t a = nullptr, b = nullptr; bool on;
+    ProfScope(cudaStream_t s, int k) : st(s), kind(k), on(g_prof_on) {
+        if (!on) return;
+        if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { on = false; return; }
+        cudaEventRecord(a, st);
+    }
+    ~ProfScope() {
+        if (!on) return;
+        cudaEventRecord(b, st);
+        std::lock_guard<std::mutex> lk(g_prof_mu);
+        g_prof.push_back({kind, a, b});
+    }
+};
+
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 void carve_scratch(const Problem& p, void* base, Scratch* s) {
@@ -112,11 +135,12 @@ static int check_ws(const Problem& p, void* ws, size_t ws_bytes, Scratch* s) {
 // steps shared by compress and query: norms + frame sums, anchor, matching + gate
 static int run_front(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                      unsigned char* keep, cudaStream_t st) {
-    cudaError_t e = launch_norm_sum(p, s, st);
+    cudaError_t e;
+    { ProfScope ps(st, PK_NORM_SUM); e = launch_norm_sum(p, s, st); }
     if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_anchor_pick(p, s, out_anchor, st);
+    { ProfScope ps(st, PK_ANCHOR_PICK); e = launch_anchor_pick(p, s, out_anchor, st); }
     if (e != cudaSuccess) return cuda_fail(e);
-    e = launch_match(p, s, shat, dst, keep, st);
+    { ProfScope ps(st, PK_MATCH); e = launch_match(p, s, shat, dst, keep, st); }
     if (e != cudaSuccess) return cuda_fail(e);
     return TTF_OK;
 }
@@ -127,7 +151,8 @@ static int compress_impl(const Problem& p, void* ws, void* out_tokens, int* out_
     carve_scratch(p, ws, &s);
     int rc = run_front(p, s, nullptr, s.shat, s.dst, s.keep, st);
     if (rc != TTF_OK) return rc;
-    cudaError_t e = launch_compact(p, s, out_tokens, out_pos, out_count, st);
+    cudaError_t e;
+    { ProfScope ps(st, PK_COMPACT); e = launch_compact(p, s, out_tokens, out_pos, out_count, st); }
     if (e != cudaSuccess) return cuda_fail(e);
     return TTF_OK;
 }
@@ -142,7 +167,8 @@ static int query_impl(const Problem& p, void* ws, int* out_anchor, unsigned char
     int rc = run_front(p, s, out_anchor, shat, dst, keep, st);
     if (rc != TTF_OK) return rc;
     if (out_fuse) {
-        cudaError_t e = launch_fuse_count(p, s, dst, keep, out_fuse, st);
+        cudaError_t e;
+        { ProfScope ps(st, PK_FUSE_COUNT); e = launch_fuse_count(p, s, dst, keep, out_fuse, st); }
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return TTF_OK;
@@ -301,6 +327,32 @@ int ttf_compress_host(const void* features_host, int F, int H, int W, int C, int
     if (e == cudaSuccess) e = cudaStreamSynchronize(st);
     if (e != cudaSuccess) return cuda_fail(e);
     return TTF_OK;
+}
+
+int ttf_profile_begin(void) {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    for (auto& r : g_prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+    g_prof.clear();
+    g_prof_on = true;
+    return TTF_OK;
+}
+
+int ttf_profile_end(double* total_ms, long long* launches, int kinds) {
+    if (!total_ms || !launches || kinds < 1) return TTF_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof_on = false;
+    for (int k = 0; k < kinds; ++k) { total_ms[k] = 0.0; launches[k] = 0; }
+    cudaError_t first = cudaSuccess;
+    for (auto& r : g_prof) {
+        float ms = 0.f;
+        cudaError_t e = cudaEventSynchronize(r.b);
+        if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, r.a, r.b);
+        if (e != cudaSuccess && first == cudaSuccess) first = e;
+        if (e == cudaSuccess && r.kind < kinds) { total_ms[r.kind] += ms; launches[r.kind] += 1; }
+        cudaEventDestroy(r.a); cudaEventDestroy(r.b);
+    }
+    g_prof.clear();
+    return first == cudaSuccess ? TTF_OK : cuda_fail(first);
 }
 
 int ttf_release(void) {

@@ -68,3 +68,17 @@ def test_null_and_nonfinite_arguments_are_rejected_before_any_launch(lib):
 
 def test_decode_alignment_helper():
     assert P.ttf_decode_pos(2703, 57, 0) == 2760 and P.ttf_decode_pos(2703, 57, 4) == 2764
+
+
+def test_flop_counter_reproduces_table3():
+    """The paper's Table 3 prints 18 / 164 / 456 MFLOPS for r = 0 / 1 / 2 (F=32, N=256); 2(F-1)N(2r+1)^2 C
+    gives those figures for C = 1152 (456 is 25 x the rounded per-candidate figure)."""
+    from paper_2605_07355_b200 import accounting as A
+    rows = [l.split() for l in open(os.path.join(ROOT, "tests", "golden", "table3_mflops.txt")) if l[0].isdigit()]
+    got = {int(r): A.matching_flops_nominal(32, 256, 1152, int(r)) / 1e6 for r, _, _ in rows}
+    for r, _, printed in rows:
+        assert abs(got[int(r)] - float(printed)) / float(printed) < 0.02
+    assert abs(got[1] / 1e3 - 0.16) < 0.01                  # abstract: about 0.16 GFLOPs
+    assert A.window_pairs(16, 16, 1) == 2116 and A.window_pairs(32, 32, 2) == 23716
+    assert A.matching_flops(32, 16, 16, 1152, 1) < A.matching_flops_nominal(32, 256, 1152, 1)
+    assert A.pass_bytes(32, 256, 4096, 2, 2703) == 32 * 256 * 4096 * 2 + 2703 * 8192 + 2703 * 12 + 4
