@@ -80,6 +80,196 @@ k_match_generic(const T* __restrict__ X, int F, int H, int W, int C, int r, floa
     }
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// bf16 fast path.  Per grid cell the work is a small dense contraction: the F source rows at that cell times
+// the (2r+1)^2 candidate anchor rows, over C channels.  At 9 to 25 multiply-adds per loaded element the plain
+// fp32 pipes, not memory, bound the per-token formulation, so the products go through the warp-level bf16
+// MMA (m16n8k16, fp32 accumulate: bf16 products are exact in fp32).  M = frames (16 per tile), N = candidates
+// (8 per tile), K = channels.
+//
+// No shared-memory staging: a dot product does not care about the order of its terms, so the K index of a
+// fragment may be any fixed permutation of the channels as long as A and B use the same one.  Each lane loads
+// 16 contiguous bytes (8 channels) of "its" row (frame g / g+8 for A, candidate g for B; g = lane/4) at
+// 16-byte column lane%4 of a 64-byte block and uses them as its fragment elements of two consecutive MMA
+// steps.  Loads are therefore 128-bit, coalesced in 64-byte runs per row, and feed the MMA directly.
+//
+// The 8 warps of a CTA take interleaved 64-byte blocks of the rows (split K) and their partial products are
+// summed through shared memory in warp order, so the result does not depend on scheduling.
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+constexpr int kMmaWarps = 8;
+
+template <int MT, int NT>
+struct MmaStage {
+    uint4 a[MT][2];
+    uint4 b[NT];
+};
+
+template <int MT, int NT>
+__device__ __forceinline__ void mma_load_stage(MmaStage<MT, NT>& sg, const uint4* const (&arow)[MT][2],
+                                               const uint4* const (&brow)[NT], const bool (&bvalid)[NT],
+                                               int idx, int units) {
+    const bool ok = idx < units;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) sg.a[mt][h] = ok ? __ldg(arow[mt][h] + idx) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) sg.b[nt] = (ok && bvalid[nt]) ? __ldg(brow[nt] + idx) : make_uint4(0, 0, 0, 0);
+}
+
+template <int MT, int NT>
+__device__ __forceinline__ void mma_compute_stage(const MmaStage<MT, NT>& sg, float (&acc)[MT][NT][4]) {
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            mma_bf16_16816(acc[mt][nt], sg.a[mt][0].x, sg.a[mt][1].x, sg.a[mt][0].y, sg.a[mt][1].y, sg.b[nt].x, sg.b[nt].y);
+            mma_bf16_16816(acc[mt][nt], sg.a[mt][0].z, sg.a[mt][1].z, sg.a[mt][0].w, sg.a[mt][1].w, sg.b[nt].z, sg.b[nt].w);
+        }
+}
+
+template <int MT, int NT>
+__global__ void __launch_bounds__(kMmaWarps * 32, 2)
+k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t, int nslice,
+            const int* __restrict__ hdr, const float* __restrict__ ssq,
+            float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep,
+            int* __restrict__ cnt)
+{
+    constexpr int FR = 16 * MT;      // frames per CTA
+    constexpr int NC = 8 * NT;       // candidate slots per CTA (>= (2r+1)^2)
+    __shared__ float s_part[kMmaWarps][FR][NC];
+    __shared__ float s_dot[FR][NC];
+    __shared__ float s_rs[FR];
+    __shared__ float s_ra[NC];
+    __shared__ int s_j[NC];
+
+    const int N = H * W;
+    const int i = blockIdx.x % N;
+    const int k0 = (blockIdx.x / N) * FR;
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    const int g = lane >> 2, tig = lane & 3;
+    const int a = hdr[HDR_ANCHOR];
+    const int y = i / W, x = i - y * W;
+    const int side = 2 * r + 1, ncand = side * side;
+    const size_t FN = (size_t)F * N;
+    const int units = C / 8;                     // 16-byte units per row
+
+    // candidate c = (dy + r) * side + (dx + r): ascending c is ascending anchor index among in-grid cells
+    auto cand_index = [&](int c) -> int {
+        if (c >= ncand) return -1;
+        const int yy = y + c / side - r, xx = x + c % side - r;
+        return (yy >= 0 && yy < H && xx >= 0 && xx < W) ? yy * W + xx : -1;
+    };
+
+    if (tid < NC) {
+        const int j = cand_index(tid);
+        s_j[tid] = j;
+        s_ra[tid] = j >= 0 ? inv_norm(ssq, nslice, FN, (size_t)a * N + j) : 0.f;
+    } else if (tid >= 64 && tid < 64 + FR) {
+        const int k = k0 + tid - 64;
+        s_rs[tid - 64] = k < F ? inv_norm(ssq, nslice, FN, (size_t)k * N + i) : 0.f;
+    }
+
+    const uint4* arow[MT][2];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int k = min(F - 1, k0 + mt * 16 + h * 8 + g);    // rows past the clip repeat the last frame
+            arow[mt][h] = reinterpret_cast<const uint4*>(X + ((size_t)k * N + i) * C);
+        }
+    const uint4* brow[NT];
+    bool bvalid[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const int j = cand_index(nt * 8 + g);
+        bvalid[nt] = j >= 0;
+        brow[nt] = reinterpret_cast<const uint4*>(X + ((size_t)a * N + (j >= 0 ? j : 0)) * C);
+    }
+
+    float acc[MT][NT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[mt][nt][q] = 0.f;
+
+    // split K: warp w takes 64-byte blocks w, w + 8, ...; two blocks are in flight per warp
+    const int nblk = (units + 3) / 4;
+    MmaStage<MT, NT> s0, s1;
+    int blk = w;
+    if (blk < nblk) mma_load_stage<MT, NT>(s0, arow, brow, bvalid, blk * 4 + tig, units);
+    for (; blk < nblk; blk += 2 * kMmaWarps) {
+        const int nb1 = blk + kMmaWarps, nb2 = blk + 2 * kMmaWarps;
+        if (nb1 < nblk) mma_load_stage<MT, NT>(s1, arow, brow, bvalid, nb1 * 4 + tig, units);
+        mma_compute_stage<MT, NT>(s0, acc);
+        if (nb1 < nblk) {
+            if (nb2 < nblk) mma_load_stage<MT, NT>(s0, arow, brow, bvalid, nb2 * 4 + tig, units);
+            mma_compute_stage<MT, NT>(s1, acc);
+        }
+    }
+
+    // accumulator fragment: c0,c1 = (frame g, candidates 2*tig, 2*tig+1); c2,c3 = (frame g+8, same candidates)
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            s_part[w][mt * 16 + g][nt * 8 + 2 * tig] = acc[mt][nt][0];
+            s_part[w][mt * 16 + g][nt * 8 + 2 * tig + 1] = acc[mt][nt][1];
+            s_part[w][mt * 16 + g + 8][nt * 8 + 2 * tig] = acc[mt][nt][2];
+            s_part[w][mt * 16 + g + 8][nt * 8 + 2 * tig + 1] = acc[mt][nt][3];
+        }
+    __syncthreads();
+    for (int idx = tid; idx < FR * NC; idx += kMmaWarps * 32) {
+        float d = 0.f;
+#pragma unroll
+        for (int ww = 0; ww < kMmaWarps; ++ww) d += (&s_part[ww][0][0])[idx];
+        (&s_dot[0][0])[idx] = d;
+    }
+    __syncthreads();
+
+    if (tid < FR) {
+        const int k = k0 + tid;
+        if (k < F) {
+            const size_t f = (size_t)k * N + i;
+            if (k == a) {                           // anchor tokens are always retained (Eq. mask)
+                shat[f] = 1.0f; dst[f] = i; keep[f] = 1;
+            } else {
+                const float rs = s_rs[tid];
+                float best = -INFINITY;
+                int best_j = -1;
+                for (int c = 0; c < ncand; ++c) {
+                    const int j = s_j[c];
+                    if (j < 0) continue;
+                    const float s = s_dot[tid][c] * rs * s_ra[c];
+                    if (s > best || best_j < 0) { best = s; best_j = j; }
+                }
+                const unsigned char kp = !(best > t);
+                shat[f] = best; dst[f] = best_j; keep[f] = kp;
+                if (kp) atomicAdd(&cnt[k], 1);
+            }
+        }
+    }
+}
+
+template <int MT, int NT>
+static cudaError_t launch_mma_t(const Problem& p, const Scratch& s, float* shat, int* dst, unsigned char* keep,
+                                cudaStream_t st) {
+    const long long chunks = (p.F + 16 * MT - 1) / (16 * MT);
+    k_match_mma<MT, NT><<<(unsigned)(chunks * p.N), kMmaWarps * 32, 0, st>>>(
+        reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t, p.nslice, s.hdr, s.ssq, shat, dst,
+        keep, s.cnt);
+    return cudaGetLastError();
+}
+
 template <typename T, int V>
 static cudaError_t launch_generic_t(const Problem& p, const Scratch& s, float* shat, int* dst,
                                     unsigned char* keep, cudaStream_t st) {
@@ -102,6 +292,11 @@ cudaError_t launch_match(const Problem& p, const Scratch& s, float* shat, int* d
                          cudaStream_t st) {
     if (p.dtype == 0) return p.vec ? launch_generic_t<float, 4>(p, s, shat, dst, keep, st)
                                    : launch_generic_t<float, 1>(p, s, shat, dst, keep, st);
+    if (p.vec && p.r <= 2 && (long long)p.N * ((p.F + 31) / 32) < (1LL << 31)) {
+        if (p.r == 0) return launch_mma_t<2, 1>(p, s, shat, dst, keep, st);
+        if (p.r == 1) return launch_mma_t<2, 2>(p, s, shat, dst, keep, st);
+        return launch_mma_t<2, 4>(p, s, shat, dst, keep, st);
+    }
     return p.vec ? launch_generic_t<bf16_t, 8>(p, s, shat, dst, keep, st)
                  : launch_generic_t<bf16_t, 1>(p, s, shat, dst, keep, st);
 }
