@@ -50,7 +50,8 @@ typedef enum {
     TTF_ERR_INVALID_ARG = 1,   /* NULL pointer, size < 1, r < 0, non-finite t, unknown dtype or option       */
     TTF_ERR_UNSUPPORTED = 2,   /* sizes beyond int32 indexing (F*H*W >= 2^31 or F*H*W*C*itemsize >= 2^46)    */
     TTF_ERR_WORKSPACE = 3,     /* caller workspace NULL, smaller than ttf_workspace_bytes or not 256-aligned */
-    TTF_ERR_CUDA = 4           /* a CUDA runtime call failed (see ttf_last_cuda_error)                       */
+    TTF_ERR_CUDA = 4,          /* a CUDA runtime call failed (see ttf_last_cuda_error)                       */
+    TTF_ERR_STATIC_LIMIT = 5   /* ttf_query_static: the clip needs more scratch than TTF_STATIC_SCRATCH_BYTES */
 } ttf_status;
 
 typedef struct CUstream_st* ttf_stream_t;      /* same type as cudaStream_t */
@@ -115,6 +116,35 @@ int ttf_query_ws(const void* features, int F, int H, int W, int C, int r, float 
  */
 int ttf_compress_host(const void* features_host, int F, int H, int W, int C, int r, float t, int dtype,
                       void* out_tokens_host, int* out_count_host, int* out_pos_thw_host);
+
+/*
+ * ttf_query for callers that must not allocate device memory.  (The paper has no counterpart: this entry
+ * point exists for the needs of the host program, not of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits or too costly -- a serving loop whose memory
+ * was handed over in full to a framework's pool at start-up, a latency-critical thread that cannot afford
+ * the device-wide synchronisation an allocation implies, a plug-in running under a host that forbids
+ * allocations after initialisation.  ttf_query allocates scratch on first use per stream and ttf_query_ws
+ * needs a buffer the caller had to get from somewhere; this variant needs neither.
+ *
+ * How: its scratch is a fixed array of TTF_STATIC_SCRATCH_BYTES (8 MiB) that is part of the library image,
+ * so every GPU on which the library is used holds those 8 MiB until the process exits, whether or not this
+ * function is ever called.  Arguments, outputs and results are exactly those of ttf_query.
+ *   - A clip whose scratch need (the unaligned-layout figure ttf_workspace_bytes reports is an upper bound;
+ *     the 8B-shaped clip F=32, 16x16, C=4096 bf16 needs about 1.3 MiB) exceeds the array is rejected with
+ *     TTF_ERR_STATIC_LIMIT before anything is launched.
+ *   - The first call on each device looks up the array's device address (a CUDA runtime query, no
+ *     allocation); make that first call outside any stream capture.  Later calls only enqueue work:
+ *     a small memset of the control words, then the kernels.
+ *   - All calls on a device share the one array and it keeps whatever the previous call left in it.  Calls
+ *     on the same stream are ordered and safe.  Two calls that can overlap on the GPU (different streams,
+ *     no event between them) race on the scratch and give undefined results: serialise them.
+ * No cudaMalloc, cudaFree or other allocating routine is called on any path of this function.
+ */
+#define TTF_STATIC_SCRATCH_BYTES (8u << 20)
+int ttf_query_static(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                     int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
+                     int* out_fuse_cnt, ttf_stream_t stream);
 
 /*
  * Per-kernel timing (the paper has no counterpart; it reports no profile of the pass).  Between

@@ -21,7 +21,9 @@ TTF_OK = 0
 EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
+    "ttf_query_static",
 ]
+TTF_STATIC_SCRATCH_BYTES = 8 << 20
 KERNEL_KINDS = ["norm_sum", "anchor_pick", "match", "compact", "frame_prefix", "fuse_count"]
 
 _lib = None
@@ -59,6 +61,8 @@ def lib() -> ctypes.CDLL:
         L.ttf_query.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp]
         L.ttf_query_ws.restype = i
         L.ttf_query_ws.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.ttf_query_static.restype = i
+        L.ttf_query_static.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp]
         L.ttf_compress_host.restype = i
         L.ttf_compress_host.argtypes = [vp] + shape + [f, i, vp, vp, vp]
         L.ttf_release.restype = i
@@ -161,6 +165,23 @@ def ttf_query(features: torch.Tensor, r: int, t: float, workspace: Optional[torc
     if rc != TTF_OK:
         raise TTFError(rc, "ttf_query")
     return {k: v for k, v in out.items() if v is not None}
+
+
+def ttf_query_static(features: torch.Tensor, r: int, t: float, out: dict, stream=None) -> dict:
+    """ttf_query_static: the query pass on the library's built-in scratch array; allocates nothing.
+
+    For callers that may not allocate: ``out`` must already hold the tensors to fill (any of "anchor" int32[1],
+    "keep" uint8[F*H*W], "dst" int32[F*H*W], "best_sim" float32[F*H*W], "fuse_cnt" int32[H*W]); this wrapper
+    creates none.  Calls that can overlap on the GPU share the scratch and race; keep them on one stream.
+    Raises TTFError(TTF_ERR_STATIC_LIMIT) when the clip needs more than TTF_STATIC_SCRATCH_BYTES."""
+    F, H, W, C = _check_features(features, "cuda")
+    args = [_p(features), F, H, W, C, int(r), float(t), _dtype_code(features), _p(out.get("anchor")),
+            _p(out.get("keep")), _p(out.get("dst")), _p(out.get("best_sim")), _p(out.get("fuse_cnt"))]
+    with torch.cuda.device(features.device):
+        rc = lib().ttf_query_static(*args, _stream_ptr(stream))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_query_static")
+    return out
 
 
 def ttf_compress_host(features: torch.Tensor, r: int, t: float, out_tokens: Optional[torch.Tensor] = None,

@@ -193,6 +193,31 @@ static cudaError_t grow(void** p, size_t* have, size_t want) {
     return e;
 }
 
+// ---- scratch of ttf_query_static: part of the library image, one copy per GPU that loads it --------------
+// In host code `g_static_scratch` is only a handle for the runtime's symbol calls, never a device address;
+// static_scratch_address() asks the runtime for the address once per device and caches it.
+static __device__ __align__(256) unsigned char g_static_scratch[TTF_STATIC_SCRATCH_BYTES];
+constexpr int kMaxStaticDevices = 64;
+static void* g_static_addr[kMaxStaticDevices] = {};
+static std::mutex g_static_mu;
+
+static int static_scratch_address(void** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (dev < 0 || dev >= kMaxStaticDevices) return TTF_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (!g_static_addr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);     // `dev` is current: the address is this device's copy
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (!p || reinterpret_cast<uintptr_t>(p) % 256 != 0) return TTF_ERR_WORKSPACE;
+        g_static_addr[dev] = p;
+    }
+    *out = g_static_addr[dev];
+    return TTF_OK;
+}
+
 }  // namespace ttf
 
 using namespace ttf;
@@ -206,6 +231,7 @@ const char* ttf_status_string(int status) {
         case TTF_ERR_UNSUPPORTED: return "TTF_ERR_UNSUPPORTED";
         case TTF_ERR_WORKSPACE: return "TTF_ERR_WORKSPACE";
         case TTF_ERR_CUDA: return "TTF_ERR_CUDA";
+        case TTF_ERR_STATIC_LIMIT: return "TTF_ERR_STATIC_LIMIT";
         default: return "TTF_ERR_UNKNOWN";
     }
 }
@@ -278,6 +304,25 @@ int ttf_query(const void* features, int F, int H, int W, int C, int r, float t, 
     void* ws = nullptr;
     rc = cached_scratch(s.bytes, (cudaStream_t)stream, &ws);
     if (rc != TTF_OK) return rc;
+    return query_impl(p, ws, out_anchor, out_keep, out_dst, out_best_sim, out_fuse_cnt, (cudaStream_t)stream);
+}
+
+int ttf_query_static(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                     int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
+                     int* out_fuse_cnt, ttf_stream_t stream) {
+    if (!features) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    Scratch s;
+    carve_scratch(p, nullptr, &s);
+    if (s.bytes > (size_t)TTF_STATIC_SCRATCH_BYTES) return TTF_ERR_STATIC_LIMIT;
+    void* ws = nullptr;
+    rc = static_scratch_address(&ws);
+    if (rc != TTF_OK) return rc;
+    // the array still holds the previous call's state: the control words must start at zero
+    cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(int) * kHdrInts, (cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e);
     return query_impl(p, ws, out_anchor, out_keep, out_dst, out_best_sim, out_fuse_cnt, (cudaStream_t)stream);
 }
 
