@@ -31,12 +31,10 @@ def pass_bytes(F: int, N: int, C: int, itemsize: int, count: int) -> int:
 def kernel_bytes(kind: str, F: int, N: int, C: int, itemsize: int, count: int, nslice: int) -> int:
     """Algorithmic bytes of one launch of each kernel kind."""
     X = F * N * C * itemsize
-    if kind == "norm_sum":          # reads X; writes frame sums and per-slice squared norms
+    if kind == "norm_anchor":       # reads X; writes frame sums and per-slice squared norms
         return X + F * C * 4 + nslice * F * N * 4
     if kind == "match":             # reads X (sources + anchor frame once); writes s_hat, dst, keep
         return X + F * N * 9
     if kind == "compact":           # reads the retained rows, writes them with their positions
         return 2 * count * C * itemsize + count * 12 + F * N + 4
-    if kind == "anchor_pick":
-        return 2 * F * C * 4
     raise KeyError(kind)

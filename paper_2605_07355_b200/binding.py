@@ -24,7 +24,7 @@ EXPORTS = [
     "ttf_query_static",
 ]
 TTF_STATIC_SCRATCH_BYTES = 8 << 20
-KERNEL_KINDS = ["norm_sum", "anchor_pick", "match", "compact", "frame_prefix", "fuse_count"]
+KERNEL_KINDS = ["norm_anchor", "match", "compact", "fuse_count"]
 
 _lib = None
 

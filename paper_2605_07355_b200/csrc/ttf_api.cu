@@ -33,8 +33,7 @@ int sm_count() {
 }
 
 // ---- optional per-kernel timing: CUDA events recorded around every launch while profiling is on ---------
-enum { PK_NORM_SUM = 0, PK_ANCHOR_PICK = 1, PK_MATCH = 2, PK_COMPACT = 3, PK_FRAME_PREFIX = 4, PK_FUSE_COUNT = 5,
-       PK_KINDS = 6 };
+enum { PK_NORM_ANCHOR = 0, PK_MATCH = 1, PK_COMPACT = 2, PK_FUSE_COUNT = 3, PK_KINDS = 4 };
 struct ProfRecord { int kind; cudaEvent_t a, b; };
 static std::mutex g_prof_mu;
 static bool g_prof_on = false;
@@ -62,12 +61,17 @@ void carve_scratch(const Problem& p, void* base, Scratch* s) {
     char* b = reinterpret_cast<char*>(base);
     auto take = [&](size_t bytes) { size_t o = off; off = align256(off + bytes); return b ? (void*)(b + o) : nullptr; };
     const size_t FN = (size_t)p.F * p.N;
-    s->hdr = (int*)take(sizeof(int) * kHdrInts);
+    // control words first, contiguous: one memset of (kHdrInts + nslice) ints clears them
+    s->hdr = (int*)take(sizeof(int) * ((size_t)kHdrInts + p.nslice));
+    s->done_slice = s->hdr ? s->hdr + kHdrInts : nullptr;
     s->cnt = (int*)take(sizeof(int) * p.F);
     s->prefix = (int*)take(sizeof(int) * ((size_t)p.F + 1));
     s->fcos = (float*)take(sizeof(float) * p.F);
-    s->g = (float*)take(sizeof(float) * p.C);
+    s->Sp = (float*)take(sizeof(float) * (size_t)norm_token_groups(p) * p.F * p.C);
     s->S = (float*)take(sizeof(float) * (size_t)p.F * p.C);
+    s->Dp = (float*)take(sizeof(float) * (size_t)p.nslice * p.F);
+    s->Qp = (float*)take(sizeof(float) * (size_t)p.nslice * p.F);
+    s->Gp = (float*)take(sizeof(float) * (size_t)p.nslice);
     s->ssq = (float*)take(sizeof(float) * (size_t)p.nslice * FN);
     s->shat = (float*)take(sizeof(float) * FN);
     s->dst = (int*)take(sizeof(int) * FN);
@@ -120,6 +124,9 @@ static int cached_scratch(size_t bytes, cudaStream_t st, void** out) {
         e = cudaMalloc(&ce.ptr, bytes);
         if (e != cudaSuccess) { ce.ptr = nullptr; return cuda_fail(e); }
         ce.bytes = bytes;
+        // the arrival counters must start at zero; the kernels leave them at zero after every call
+        e = cudaMemsetAsync(ce.ptr, 0, bytes, st);
+        if (e != cudaSuccess) return cuda_fail(e);
     }
     *out = ce.ptr;
     return TTF_OK;
@@ -132,13 +139,17 @@ static int check_ws(const Problem& p, void* ws, size_t ws_bytes, Scratch* s) {
     return TTF_OK;
 }
 
+// Scratch that is not the library's own may hold anything: clear the control words (stream-ordered).
+static int clear_control(const Problem& p, void* ws, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(int) * ((size_t)kHdrInts + p.nslice), st);
+    return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+}
+
 // steps shared by compress and query: norms + frame sums, anchor, matching + gate
 static int run_front(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                      unsigned char* keep, cudaStream_t st) {
     cudaError_t e;
-    { ProfScope ps(st, PK_NORM_SUM); e = launch_norm_sum(p, s, st); }
-    if (e != cudaSuccess) return cuda_fail(e);
-    { ProfScope ps(st, PK_ANCHOR_PICK); e = launch_anchor_pick(p, s, out_anchor, st); }
+    { ProfScope ps(st, PK_NORM_ANCHOR); e = launch_norm_anchor(p, s, out_anchor, st); }
     if (e != cudaSuccess) return cuda_fail(e);
     { ProfScope ps(st, PK_MATCH); e = launch_match(p, s, shat, dst, keep, st); }
     if (e != cudaSuccess) return cuda_fail(e);
@@ -247,7 +258,12 @@ int ttf_workspace_bytes(int F, int H, int W, int C, int r, int dtype, size_t* by
     if (rc != TTF_OK) return rc;
     Scratch s;
     carve_scratch(p, nullptr, &s);
-    *bytes = s.bytes;
+    size_t need = s.bytes;
+    rc = make_problem(reinterpret_cast<const void*>(uintptr_t(256)), F, H, W, C, r, 0.f, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    carve_scratch(p, nullptr, &s);
+    if (s.bytes > need) need = s.bytes;
+    *bytes = need;
     return TTF_OK;
 }
 
@@ -260,6 +276,8 @@ int ttf_compress_ws(const void* features, int F, int H, int W, int C, int r, flo
     if (rc != TTF_OK) return rc;
     Scratch s;
     rc = check_ws(p, workspace, workspace_bytes, &s);
+    if (rc != TTF_OK) return rc;
+    rc = clear_control(p, workspace, (cudaStream_t)stream);
     if (rc != TTF_OK) return rc;
     return compress_impl(p, workspace, out_tokens, out_count, out_pos_thw, (cudaStream_t)stream);
 }
@@ -287,6 +305,8 @@ int ttf_query_ws(const void* features, int F, int H, int W, int C, int r, float 
     if (rc != TTF_OK) return rc;
     Scratch s;
     rc = check_ws(p, workspace, workspace_bytes, &s);
+    if (rc != TTF_OK) return rc;
+    rc = clear_control(p, workspace, (cudaStream_t)stream);
     if (rc != TTF_OK) return rc;
     return query_impl(p, workspace, out_anchor, out_keep, out_dst, out_best_sim, out_fuse_cnt,
                       (cudaStream_t)stream);
@@ -321,8 +341,8 @@ int ttf_query_static(const void* features, int F, int H, int W, int C, int r, fl
     rc = static_scratch_address(&ws);
     if (rc != TTF_OK) return rc;
     // the array still holds the previous call's state: the control words must start at zero
-    cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(int) * kHdrInts, (cudaStream_t)stream);
-    if (e != cudaSuccess) return cuda_fail(e);
+    rc = clear_control(p, ws, (cudaStream_t)stream);
+    if (rc != TTF_OK) return rc;
     return query_impl(p, ws, out_anchor, out_keep, out_dst, out_best_sim, out_fuse_cnt, (cudaStream_t)stream);
 }
 

@@ -5,15 +5,14 @@
 // in flat (k, i) order.  That exclusive prefix is taken in two levels: the per-frame survivor counts written
 // by the matching kernel are scanned by every CTA (shared memory, or a pre-scanned array for very long
 // clips), and inside a frame the rank is a population count over the frame's keep flags.  The gather is then
-// driven from the OUTPUT side: work item (output row j, 2 KB part of the row) -> rank/select finds the source
-// row, so every warp copies the same number of bytes no matter how unevenly the survivors are spread over
-// the frames.  No CTA ever waits for another one.
+// driven from the OUTPUT side: every CTA owns an equal, contiguous range of output rows, finds their source
+// rows by rank/select and copies them, so the bytes per CTA are the same no matter how unevenly the
+// survivors are spread over the frames.  No CTA ever waits for another one.
 #include "ttf_internal.cuh"
 
 namespace ttf {
 
 constexpr int kCopyWarps = 8;
-constexpr int kPartBytes = 2048;     // bytes of one row handled by one warp-level work item
 
 // exclusive scan of the effective per-frame counts (anchor frame counts as 0) for clips with more frames
 // than fit the shared-memory scan of the gather kernel
@@ -62,13 +61,53 @@ template <> struct CopyUnit<16> { using type = uint4; };
 template <> struct CopyUnit<4> { using type = uint32_t; };
 template <> struct CopyUnit<2> { using type = uint16_t; };
 
+constexpr int kRowsPerPass = 32;     // output rows whose sources a CTA resolves before copying them
+constexpr int kCopyUnroll = 8;       // copy units in flight per thread
+
+// Cell index of the n-th (0-based) retained token of one frame: a warp-wide rank/select over the keep flags.
+// All lanes must call with the same arguments; returns -1 if the frame holds fewer than n+1 retained tokens.
+__device__ __forceinline__ int select_in_frame(const unsigned char* __restrict__ kf, int N, int n, int lane) {
+    for (int b = 0; b < N; b += 256) {                     // 8 cells per lane, 256 per step
+        const int c0 = b + lane * 8;
+        unsigned bits = 0;
+        if (c0 + 8 <= N && ((reinterpret_cast<uintptr_t>(kf + c0) & 7) == 0)) {
+            const uint2 v = *reinterpret_cast<const uint2*>(kf + c0);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                bits |= ((v.x >> (8 * e)) & 0xffu) ? (1u << e) : 0u;
+                bits |= ((v.y >> (8 * e)) & 0xffu) ? (1u << (4 + e)) : 0u;
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) bits |= (c0 + e < N && kf[c0 + e] != 0) ? (1u << e) : 0u;
+        }
+        const int mine = __popc(bits);
+        int incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
+        if (n < total) {
+            const int excl = incl - mine;
+            const bool here = n >= excl && n < incl;       // exactly one lane
+            const int cell = here ? c0 + (int)__fns(bits, 0, n - excl + 1) : 0;
+            const unsigned who = __ballot_sync(0xffffffffu, here);
+            return __shfl_sync(0xffffffffu, cell, __ffs(who) - 1);
+        }
+        n -= total;
+    }
+    return -1;
+}
+
 template <int COPY_BYTES>
 __global__ void __launch_bounds__(kCopyWarps * 32)
 k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, int W, int r,
           const int* __restrict__ hdr, const int* __restrict__ cnt, const int* __restrict__ gprefix,
           const unsigned char* __restrict__ keep, const int* __restrict__ dst,
           unsigned char* __restrict__ out_tokens, int* __restrict__ out_pos, int* __restrict__ out_count,
-          int* __restrict__ fuse_cnt, int ncopy_blocks, int parts_per_row)
+          int* __restrict__ fuse_cnt, int ncopy_blocks)
 {
     using U = typename CopyUnit<COPY_BYTES>::type;
     const int N = H * W;
@@ -100,6 +139,7 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
     // ---- exclusive prefix of preserved tokens per frame ------------------------------------------------
     __shared__ int s_pre[kSmemPrefixMaxF + 1];
     __shared__ int s_warp[kCopyWarps];
+    __shared__ int s_src[kRowsPerPass];
     const int* pre;
     if (F <= kSmemPrefixMaxF) {
         // each thread scans a contiguous run of frames, runs are combined over the block in thread order
@@ -129,48 +169,54 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
     const int L = N + P;                                   // L' = N + P (Eq. Lpre)
     if (blockIdx.x == 0 && tid == 0) { *out_count = L; }
 
-    // ---- output-driven gather ---------------------------------------------------------------------------
-    const long long items = (long long)L * parts_per_row;
-    const long long stride = (long long)ncopy_blocks * kCopyWarps;
-    const int units_per_row = (int)(row_bytes / COPY_BYTES);
-    const int units_per_part = kPartBytes / COPY_BYTES;
-    for (long long it = (long long)blockIdx.x * kCopyWarps + w; it < items; it += stride) {
-        const int j = (int)(it / parts_per_row);
-        const int part = (int)(it - (long long)j * parts_per_row);
-        int k, i;
-        if (j < N) { k = a; i = j; }                        // anchor rows first (Eq. xprime_stack)
-        else {
-            const int e = j - N;
-            int lo = 0, hi = F;                             // largest k with pre[k] <= e
-            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (pre[mid] <= e) lo = mid; else hi = mid; }
-            k = lo;
-            int n = e - pre[k];                             // rank inside frame k
-            const unsigned char* kf = keep + (size_t)k * N;
-            i = -1;
-            for (int b = 0; b < N; b += 32) {
-                const int ii = b + lane;
-                const unsigned m = __ballot_sync(0xffffffffu, ii < N && kf[ii] != 0);
-                const int c = __popc(m);
-                if (n < c) { i = b + (int)__fns(m, 0, n + 1); break; }
-                n -= c;
+    // ---- output-driven gather: this CTA owns a contiguous, balanced range of output rows ------------------
+    const int j_begin = (int)((long long)L * blockIdx.x / ncopy_blocks);
+    const int j_end = (int)((long long)L * (blockIdx.x + 1) / ncopy_blocks);
+    const int upr = (int)(row_bytes / COPY_BYTES);         // copy units per row
+    for (int jb = j_begin; jb < j_end; jb += kRowsPerPass) {
+        const int rows = min(kRowsPerPass, j_end - jb);
+        __syncthreads();                                   // previous pass has finished with s_src
+        // a) source token of every output row of the pass: one warp per row
+        for (int rr = w; rr < rows; rr += kCopyWarps) {
+            const int j = jb + rr;
+            int f;
+            if (j < N) f = a * N + j;                      // anchor rows first (Eq. xprime_stack)
+            else {
+                const int e = j - N;
+                int lo = 0, hi = F;                        // largest k with pre[k] <= e
+                while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (pre[mid] <= e) lo = mid; else hi = mid; }
+                const int i = select_in_frame(keep + (size_t)lo * N, N, e - pre[lo], lane);
+                f = i < 0 ? -1 : lo * N + i;               // -1 cannot happen when cnt matches keep
             }
-            if (i < 0) continue;                            // cannot happen when cnt matches keep
+            if (lane == 0) s_src[rr] = f;
+            if (lane < 3 && f >= 0) {                      // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
+                const int k = f / N, i = f - k * N, yy = i / W;
+                out_pos[(size_t)j * 3 + lane] = lane == 0 ? k : (lane == 1 ? yy : i - yy * W);
+            }
         }
-        const size_t f = (size_t)k * N + i;
-        const U* src = reinterpret_cast<const U*>(X + f * row_bytes);
-        U* dsto = reinterpret_cast<U*>(out_tokens + (size_t)j * row_bytes);
-        const int u0 = part * units_per_part;
-        const int u1 = min(units_per_row, u0 + units_per_part);
-        for (int u = u0 + lane; u < u1; u += 32 * 4) {
-            U v[4];
+        __syncthreads();
+        // b) copy: consecutive threads move consecutive 16-byte units, several rows in flight per thread
+        const long long total = (long long)rows * upr;
+        for (long long base = tid; base < total; base += (long long)kCopyWarps * 32 * kCopyUnroll) {
+            U v[kCopyUnroll];
+            long long o[kCopyUnroll];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) if (u + q * 32 < u1) v[q] = src[u + q * 32];
+            for (int q = 0; q < kCopyUnroll; ++q) {
+                const long long u = base + (long long)q * kCopyWarps * 32;
+                o[q] = -1;
+                if (u < total) {
+                    const int rr = (int)(u / upr);
+                    const int off = (int)(u - (long long)rr * upr);
+                    const int f = s_src[rr];
+                    if (f >= 0) {
+                        v[q] = __ldcs(reinterpret_cast<const U*>(X + (size_t)f * row_bytes) + off);
+                        o[q] = (long long)(jb + rr) * upr + off;
+                    }
+                }
+            }
 #pragma unroll
-            for (int q = 0; q < 4; ++q) if (u + q * 32 < u1) dsto[u + q * 32] = v[q];
-        }
-        if (part == 0 && lane < 3) {                        // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
-            const int yy = i / W;
-            out_pos[(size_t)j * 3 + lane] = lane == 0 ? k : (lane == 1 ? yy : i - yy * W);
+            for (int q = 0; q < kCopyUnroll; ++q)
+                if (o[q] >= 0) __stcs(reinterpret_cast<U*>(out_tokens) + o[q], v[q]);
         }
     }
 }
@@ -181,7 +227,7 @@ cudaError_t launch_fuse_count(const Problem& p, const Scratch& s, const int* dst
     const int nb = (p.N + kCopyWarps - 1) / kCopyWarps;
     k_compact<4><<<nb < 1024 ? nb : 1024, kCopyWarps * 32, 0, st>>>(
         nullptr, 0, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix, keep, dst, nullptr, nullptr, nullptr,
-        fuse_cnt, 0, 1);
+        fuse_cnt, 0);
     return cudaGetLastError();
 }
 
@@ -195,7 +241,6 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    const int parts = (int)((row_bytes + kPartBytes - 1) / kPartBytes);
     const int ncopy = 2 * sm_count();
     int nfuse = (p.N + kCopyWarps - 1) / kCopyWarps;
     if (nfuse > sm_count()) nfuse = sm_count();
@@ -204,13 +249,13 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
     unsigned char* out = reinterpret_cast<unsigned char*>(out_tokens);
     if (vec)
         k_compact<16><<<grid, kCopyWarps * 32, 0, st>>>(X, row_bytes, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix,
-            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy, parts);
+            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy);
     else if (esize == 4)
         k_compact<4><<<grid, kCopyWarps * 32, 0, st>>>(X, row_bytes, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix,
-            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy, parts);
+            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy);
     else
         k_compact<2><<<grid, kCopyWarps * 32, 0, st>>>(X, row_bytes, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix,
-            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy, parts);
+            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy);
     return cudaGetLastError();
 }
 

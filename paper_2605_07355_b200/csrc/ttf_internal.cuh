@@ -13,7 +13,7 @@ constexpr int kSmemPrefixMaxF = 2048;  // frame counts up to this are scanned in
 constexpr int kHdrInts = 64;
 
 // header words of the scratch block
-enum { HDR_ANCHOR = 0, HDR_COUNT = 1, HDR_DONE0 = 2, HDR_DONE1 = 3 };
+enum { HDR_ANCHOR = 0, HDR_DONE_ALL = 1 };
 
 // Problem description handed to every launcher.
 struct Problem {
@@ -31,12 +31,16 @@ struct Problem {
 
 // Device pointers carved out of one scratch allocation.
 struct Scratch {
-    int* hdr;           // [kHdrInts]
+    int* hdr;           // [kHdrInts]  anchor frame, arrival counter of the slices
+    int* done_slice;    // [nslice]    arrival counters of the CTAs of a channel slice (directly after hdr)
     int* cnt;           // [F]   preserved tokens per source frame (Eq. gating summed over a frame)
     int* prefix;        // [F+1] exclusive scan of cnt, only used when F > kSmemPrefixMaxF
     float* fcos;        // [F]   cosine of each frame mean to the global mean (Eq. auto_anchor)
-    float* g;           // [C]   sum of all tokens
+    float* Sp;          // [TG, F, C] per-frame channel sums of each token group
     float* S;           // [F, C] per-frame channel sums
+    float* Dp;          // [nslice, F] per-slice share of <S_k, g>
+    float* Qp;          // [nslice, F] per-slice share of |S_k|^2
+    float* Gp;          // [nslice]    per-slice share of |g|^2
     float* ssq;         // [nslice, F*N] partial squared norms per channel slice
     float* shat;        // [F*N] best similarity (Eq. argmax)
     int* dst;           // [F*N] best anchor cell (Eq. dst)
@@ -49,8 +53,8 @@ struct Scratch {
 void carve_scratch(const Problem& p, void* base, Scratch* s);
 
 // Kernel launchers (each enqueues on `st` and returns the launch error, if any).
-cudaError_t launch_norm_sum(const Problem& p, const Scratch& s, cudaStream_t st);
-cudaError_t launch_anchor_pick(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st);
+int norm_token_groups(const Problem& p);   // token groups per frame of the norm/anchor sweep (shape-only rule)
+cudaError_t launch_norm_anchor(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st);
 cudaError_t launch_match(const Problem& p, const Scratch& s, float* shat, int* dst, unsigned char* keep,
                          cudaStream_t st);
 cudaError_t launch_fuse_count(const Problem& p, const Scratch& s, const int* dst, const unsigned char* keep,
@@ -72,26 +76,39 @@ __device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u 
 
 // Loads V consecutive channels starting at p (p is 16-byte aligned when V > 1) and widens them to fp32.
 template <typename T, int V> struct Loader;
+// load_raw fetches the bits (so that several loads can be in flight before any is unpacked), unpack widens.
 template <> struct Loader<float, 4> {
-    static __device__ __forceinline__ void load(const float* p, float (&x)[4]) {
-        float4 v = __ldg(reinterpret_cast<const float4*>(p));
-        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
-    }
+    using Raw = float4;
+    static __device__ __forceinline__ Raw load_raw(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+    static __device__ __forceinline__ Raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+    static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[4]) { x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+    static __device__ __forceinline__ void load(const float* p, float (&x)[4]) { unpack(load_raw(p), x); }
 };
 template <> struct Loader<float, 1> {
+    using Raw = float;
+    static __device__ __forceinline__ Raw load_raw(const float* p) { return __ldg(p); }
+    static __device__ __forceinline__ Raw zero() { return 0.f; }
+    static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[1]) { x[0] = v; }
     static __device__ __forceinline__ void load(const float* p, float (&x)[1]) { x[0] = __ldg(p); }
 };
 template <> struct Loader<bf16_t, 8> {
-    static __device__ __forceinline__ void load(const bf16_t* p, float (&x)[8]) {
-        uint4 v = __ldg(reinterpret_cast<const uint4*>(p));
+    using Raw = uint4;
+    static __device__ __forceinline__ Raw load_raw(const bf16_t* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+    static __device__ __forceinline__ Raw zero() { return make_uint4(0, 0, 0, 0); }
+    static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[8]) {
         x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);
         x[4] = bf16_lo(v.z); x[5] = bf16_hi(v.z); x[6] = bf16_lo(v.w); x[7] = bf16_hi(v.w);
     }
+    static __device__ __forceinline__ void load(const bf16_t* p, float (&x)[8]) { unpack(load_raw(p), x); }
 };
 template <> struct Loader<bf16_t, 1> {
-    static __device__ __forceinline__ void load(const bf16_t* p, float (&x)[1]) {
-        x[0] = __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
+    using Raw = float;
+    static __device__ __forceinline__ Raw load_raw(const bf16_t* p) {
+        return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
     }
+    static __device__ __forceinline__ Raw zero() { return 0.f; }
+    static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[1]) { x[0] = v; }
+    static __device__ __forceinline__ void load(const bf16_t* p, float (&x)[1]) { x[0] = load_raw(p); }
 };
 
 __device__ __forceinline__ float warp_sum(float v) {
