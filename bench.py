@@ -41,6 +41,7 @@ def parse_args():
     ap.add_argument("--clips", type=int, default=16, help="distinct clips per step (batch)")
     ap.add_argument("--streams", type=int, default=1, help="CUDA streams the clips of a step are spread over")
     ap.add_argument("--threshold", type=float, default=None)
+    ap.add_argument("--anchor", default="auto", choices=["auto", "first", "last"], help="anchor rule")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -190,10 +191,10 @@ def reference_arm(args):
     print(json.dumps(line), flush=True)
 
 
-def workload_config(spec, t, clips_per_step, streams, tokens_per_step):
+def workload_config(spec, t, clips_per_step, streams, tokens_per_step, anchor="auto"):
     return {"workload": f"{spec.name}: F={spec.F} {spec.H}x{spec.W} C={spec.C} {spec.dtype} r={spec.r} t={t:.2f}",
             "generator": spec.family, "clips_per_step": clips_per_step, "tokens_per_step": tokens_per_step,
-            "streams": streams,
+            "streams": streams, "anchor": anchor,
             "l2": "inputs rotate through a batch larger than L2; every clip starts cold in HBM"}
 
 
@@ -251,16 +252,20 @@ def main():
     fork = torch.cuda.Event()
     joins = [torch.cuda.Event() for _ in streams]
 
+    amode = {"auto": 0, "first": 1, "last": 2}[args.anchor]
+
     def step():
         if nstreams == 1:
             for j in range(nclips):
-                P.ttf_compress(devX[j], spec.r, t, out_tok[j], out_cnt[j], out_pos[j], stream=main_stream)
+                P.ttf_compress(devX[j], spec.r, t, out_tok[j], out_cnt[j], out_pos[j], stream=main_stream,
+                               anchor_mode=amode)
             return
         fork.record(main_stream)
         for s in streams:
             s.wait_event(fork)
         for j in range(nclips):
-            P.ttf_compress(devX[j], spec.r, t, out_tok[j], out_cnt[j], out_pos[j], stream=streams[j % nstreams])
+            P.ttf_compress(devX[j], spec.r, t, out_tok[j], out_cnt[j], out_pos[j], stream=streams[j % nstreams],
+                           anchor_mode=amode)
         for s, ev in zip(streams, joins):
             ev.record(s)
             main_stream.wait_event(ev)
@@ -317,8 +322,7 @@ def main():
     dominant = max(kern, key=lambda k: prof[k][0])
     peak_gbs, peak_kind = peaks()
     avg_count = sum(counts) / nclips
-    nslice = (C + 32 * (16 // spec.itemsize) - 1) // (32 * (16 // spec.itemsize))
-    kbytes = A.kernel_bytes(dominant, spec.F, spec.N, C, spec.itemsize, int(round(avg_count)), nslice)
+    kbytes = A.kernel_bytes(dominant, spec.F, spec.N, C, spec.itemsize, int(round(avg_count)))
     achieved = kbytes / (kern[dominant]["us_per_launch"] * 1e-6) / 1e9
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
                 "frac": achieved / peak_gbs, "peak_source": f"of {peak_kind}", "traffic": None,
@@ -368,7 +372,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(spec, t, nclips, nstreams, tokens_step),
+            "config": workload_config(spec, t, nclips, nstreams, tokens_step, args.anchor),
             "clips_per_s": clips_per_s, "rho": rho, "count_mean": avg_count,
             "roofline": roofline, "pass_roofline": pass_roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches_per_step * args.steps), "gpu_launches_per_step": int(launches_per_step),

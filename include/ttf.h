@@ -54,6 +54,10 @@ typedef enum {
     TTF_ERR_STATIC_LIMIT = 5   /* ttf_query_static: the clip needs more scratch than TTF_STATIC_SCRATCH_BYTES */
 } ttf_status;
 
+/* anchor rule: Eq. (auto_anchor), or the fixed first / last frame anchors compared in Table 1 and ablation A2,
+ * or an explicit frame (e.g. the rolling anchor of a streaming segment, Sec. 5 D3) */
+typedef enum { TTF_ANCHOR_AUTO = 0, TTF_ANCHOR_FIRST = 1, TTF_ANCHOR_LAST = 2, TTF_ANCHOR_EXPLICIT = 3 } ttf_anchor_mode;
+
 typedef struct CUstream_st* ttf_stream_t;      /* same type as cudaStream_t */
 
 /* Human-readable name of a ttf_status. Never NULL. */
@@ -107,6 +111,20 @@ int ttf_query(const void* features, int F, int H, int W, int C, int r, float t, 
 int ttf_query_ws(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
                  int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
                  int* out_fuse_cnt, void* workspace, size_t workspace_bytes, ttf_stream_t stream);
+
+/*
+ * ttf_compress / ttf_query with the anchor rule chosen by the caller (Table 1 rows "first", "last", "auto";
+ * ablation A2).  anchor_mode is a ttf_anchor_mode; anchor_frame is used only by TTF_ANCHOR_EXPLICIT and must
+ * lie in [0, F).  With a fixed anchor the frame-mean cosines of Eq. (auto_anchor) are not evaluated.
+ * Everything else is as in ttf_compress / ttf_query (scratch from the per-stream cache).
+ */
+int ttf_compress_ex(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                    int anchor_mode, int anchor_frame,
+                    void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream);
+int ttf_query_ex(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                 int anchor_mode, int anchor_frame,
+                 int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
+                 int* out_fuse_cnt, ttf_stream_t stream);
 
 /*
  * The same pass for callers whose tensors live in HOST memory (all four pointers are host pointers; pinned

@@ -5,7 +5,7 @@ from . import clips  # noqa: F401  (seeded synthetic clips; no method arithmetic
 
 
 def __getattr__(name):
-    if name.startswith("ttf_") or name in ("TTFError", "lib", "LIB_PATH", "EXPORTS", "KERNEL_KINDS", "TTF_STATIC_SCRATCH_BYTES", "TTF_DTYPE_F32", "TTF_DTYPE_BF16"):
+    if name.startswith(("ttf_", "TTF_")) or name in ("TTFError", "lib", "LIB_PATH", "EXPORTS", "KERNEL_KINDS", "TTF_STATIC_SCRATCH_BYTES", "TTF_DTYPE_F32", "TTF_DTYPE_BF16"):
         from . import binding
         return getattr(binding, name)
     raise AttributeError(name)

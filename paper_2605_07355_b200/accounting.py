@@ -28,11 +28,11 @@ def pass_bytes(F: int, N: int, C: int, itemsize: int, count: int) -> int:
     return F * N * C * itemsize + count * C * itemsize + count * 12 + 4
 
 
-def kernel_bytes(kind: str, F: int, N: int, C: int, itemsize: int, count: int, nslice: int) -> int:
+def kernel_bytes(kind: str, F: int, N: int, C: int, itemsize: int, count: int) -> int:
     """Algorithmic bytes of one launch of each kernel kind."""
     X = F * N * C * itemsize
-    if kind == "norm_anchor":       # reads X; writes frame sums and per-slice squared norms
-        return X + F * C * 4 + nslice * F * N * 4
+    if kind == "norm_anchor":       # reads X; writes the frame sums and one squared norm per token
+        return X + F * C * 4 + F * N * 4
     if kind == "match":             # reads X (sources + anchor frame once); writes s_hat, dst, keep
         return X + F * N * 9
     if kind == "compact":           # reads the retained rows, writes them with their positions

@@ -21,8 +21,9 @@ TTF_OK = 0
 EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
-    "ttf_query_static",
+    "ttf_query_static", "ttf_compress_ex", "ttf_query_ex",
 ]
+TTF_ANCHOR_AUTO, TTF_ANCHOR_FIRST, TTF_ANCHOR_LAST, TTF_ANCHOR_EXPLICIT = 0, 1, 2, 3
 TTF_STATIC_SCRATCH_BYTES = 8 << 20
 KERNEL_KINDS = ["norm_anchor", "match", "compact", "fuse_count"]
 
@@ -61,6 +62,10 @@ def lib() -> ctypes.CDLL:
         L.ttf_query.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp]
         L.ttf_query_ws.restype = i
         L.ttf_query_ws.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.ttf_compress_ex.restype = i
+        L.ttf_compress_ex.argtypes = [vp] + shape + [f, i, i, i, vp, vp, vp, vp]
+        L.ttf_query_ex.restype = i
+        L.ttf_query_ex.argtypes = [vp] + shape + [f, i, i, i, vp, vp, vp, vp, vp, vp]
         L.ttf_query_static.restype = i
         L.ttf_query_static.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp]
         L.ttf_compress_host.restype = i
@@ -115,8 +120,9 @@ def ttf_workspace_bytes(F: int, H: int, W: int, C: int, r: int, dtype: int) -> i
 
 def ttf_compress(features: torch.Tensor, r: int, t: float, out_tokens: Optional[torch.Tensor] = None,
                  out_count: Optional[torch.Tensor] = None, out_pos_thw: Optional[torch.Tensor] = None,
-                 workspace: Optional[torch.Tensor] = None, stream=None):
-    """ttf_compress / ttf_compress_ws.  Returns (out_tokens [F*H*W, C], out_count int32[1],
+                 workspace: Optional[torch.Tensor] = None, stream=None,
+                 anchor_mode: int = 0, anchor_frame: int = 0):
+    """ttf_compress / ttf_compress_ws (ttf_compress_ex when an anchor rule other than auto is given).  Returns (out_tokens [F*H*W, C], out_count int32[1],
     out_pos_thw int32 [F*H*W, 3]); only the first out_count rows are defined.  Does not synchronise."""
     F, H, W, C = _check_features(features, "cuda")
     dev = features.device
@@ -129,7 +135,13 @@ def ttf_compress(features: torch.Tensor, r: int, t: float, out_tokens: Optional[
         out_pos_thw = torch.empty((n, 3), dtype=torch.int32, device=dev)
     with torch.cuda.device(dev):
         sp = _stream_ptr(stream)
-        if workspace is None:
+        if anchor_mode != 0:
+            if workspace is not None:
+                raise ValueError("a fixed anchor rule uses the library's own scratch")
+            rc = lib().ttf_compress_ex(_p(features), F, H, W, C, int(r), float(t), _dtype_code(features),
+                                       int(anchor_mode), int(anchor_frame),
+                                       _p(out_tokens), _p(out_count), _p(out_pos_thw), sp)
+        elif workspace is None:
             rc = lib().ttf_compress(_p(features), F, H, W, C, int(r), float(t), _dtype_code(features),
                                     _p(out_tokens), _p(out_count), _p(out_pos_thw), sp)
         else:
@@ -142,8 +154,9 @@ def ttf_compress(features: torch.Tensor, r: int, t: float, out_tokens: Optional[
 
 
 def ttf_query(features: torch.Tensor, r: int, t: float, workspace: Optional[torch.Tensor] = None, stream=None,
-              want=("anchor", "keep", "dst", "best_sim", "fuse_cnt")) -> dict:
-    """ttf_query / ttf_query_ws.  Returns the requested device tensors.  Does not synchronise."""
+              want=("anchor", "keep", "dst", "best_sim", "fuse_cnt"), anchor_mode: int = 0,
+              anchor_frame: int = 0) -> dict:
+    """ttf_query / ttf_query_ws (ttf_query_ex when an anchor rule other than auto is given).  Returns the requested device tensors.  Does not synchronise."""
     F, H, W, C = _check_features(features, "cuda")
     dev = features.device
     n = F * H * W
@@ -158,7 +171,11 @@ def ttf_query(features: torch.Tensor, r: int, t: float, workspace: Optional[torc
             _p(out["dst"]), _p(out["best_sim"]), _p(out["fuse_cnt"])]
     with torch.cuda.device(dev):
         sp = _stream_ptr(stream)
-        if workspace is None:
+        if anchor_mode != 0:
+            if workspace is not None:
+                raise ValueError("a fixed anchor rule uses the library's own scratch")
+            rc = lib().ttf_query_ex(*args[:8], int(anchor_mode), int(anchor_frame), *args[8:], sp)
+        elif workspace is None:
             rc = lib().ttf_query(*args, sp)
         else:
             rc = lib().ttf_query_ws(*args, _p(workspace), workspace.numel() * workspace.element_size(), sp)

@@ -61,17 +61,15 @@ void carve_scratch(const Problem& p, void* base, Scratch* s) {
     char* b = reinterpret_cast<char*>(base);
     auto take = [&](size_t bytes) { size_t o = off; off = align256(off + bytes); return b ? (void*)(b + o) : nullptr; };
     const size_t FN = (size_t)p.F * p.N;
-    // control words first, contiguous: one memset of (kHdrInts + nslice) ints clears them
-    s->hdr = (int*)take(sizeof(int) * ((size_t)kHdrInts + p.nslice));
-    s->done_slice = s->hdr ? s->hdr + kHdrInts : nullptr;
+    s->hdr = (int*)take(sizeof(int) * kHdrInts);      // control words first: one small memset clears them
     s->cnt = (int*)take(sizeof(int) * p.F);
     s->prefix = (int*)take(sizeof(int) * ((size_t)p.F + 1));
     s->fcos = (float*)take(sizeof(float) * p.F);
     s->Sp = (float*)take(sizeof(float) * (size_t)norm_token_groups(p) * p.F * p.C);
     s->S = (float*)take(sizeof(float) * (size_t)p.F * p.C);
-    s->Dp = (float*)take(sizeof(float) * (size_t)p.nslice * p.F);
-    s->Qp = (float*)take(sizeof(float) * (size_t)p.nslice * p.F);
-    s->Gp = (float*)take(sizeof(float) * (size_t)p.nslice);
+    s->Dp = (float*)take(sizeof(float) * (size_t)p.nsl * p.F);
+    s->Qp = (float*)take(sizeof(float) * (size_t)p.nsl * p.F);
+    s->Gp = (float*)take(sizeof(float) * (size_t)p.nsl);
     s->ssq = (float*)take(sizeof(float) * (size_t)p.nslice * FN);
     s->shat = (float*)take(sizeof(float) * FN);
     s->dst = (int*)take(sizeof(int) * FN);
@@ -95,9 +93,11 @@ static int make_problem(const void* X, int F, int H, int W, int C, int r, float 
     const long long row_bytes = (long long)C * esize;
     p->vec = (row_bytes % 16 == 0) && (reinterpret_cast<uintptr_t>(X) % 16 == 0);
     p->lanes_elems = p->vec ? (int)(16 / esize) : 1;
-    const long long per_slice = 32LL * p->lanes_elems;
-    p->nslice = (int)((C + per_slice - 1) / per_slice);
-    if ((long long)F * p->nslice >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
+    const long long chunks = ((long long)C + p->lanes_elems - 1) / p->lanes_elems;
+    p->cpt = chunks <= 256 ? 1 : 2;
+    p->ncb = (int)((chunks + 256LL * p->cpt - 1) / (256LL * p->cpt));
+    p->nslice = 8 * p->ncb;
+    p->nsl = C % 4 == 0 ? (C + 255) / 256 : (C + 31) / 32;
     p->anchor_mode = 0; p->anchor_arg = 0;
     return TTF_OK;
 }
@@ -140,8 +140,8 @@ static int check_ws(const Problem& p, void* ws, size_t ws_bytes, Scratch* s) {
 }
 
 // Scratch that is not the library's own may hold anything: clear the control words (stream-ordered).
-static int clear_control(const Problem& p, void* ws, cudaStream_t st) {
-    cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(int) * ((size_t)kHdrInts + p.nslice), st);
+static int clear_control(const Problem&, void* ws, cudaStream_t st) {
+    cudaError_t e = cudaMemsetAsync(ws, 0, sizeof(int) * kHdrInts, st);
     return e == cudaSuccess ? TTF_OK : cuda_fail(e);
 }
 
@@ -318,6 +318,47 @@ int ttf_query(const void* features, int F, int H, int W, int C, int r, float t, 
     if (!features) return TTF_ERR_INVALID_ARG;
     Problem p;
     int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    Scratch s;
+    carve_scratch(p, nullptr, &s);
+    void* ws = nullptr;
+    rc = cached_scratch(s.bytes, (cudaStream_t)stream, &ws);
+    if (rc != TTF_OK) return rc;
+    return query_impl(p, ws, out_anchor, out_keep, out_dst, out_best_sim, out_fuse_cnt, (cudaStream_t)stream);
+}
+
+static int set_anchor_rule(Problem* p, int anchor_mode, int anchor_frame) {
+    if (anchor_mode < TTF_ANCHOR_AUTO || anchor_mode > TTF_ANCHOR_EXPLICIT) return TTF_ERR_INVALID_ARG;
+    if (anchor_mode == TTF_ANCHOR_EXPLICIT && (anchor_frame < 0 || anchor_frame >= p->F)) return TTF_ERR_INVALID_ARG;
+    p->anchor_mode = anchor_mode;
+    p->anchor_arg = anchor_mode == TTF_ANCHOR_EXPLICIT ? anchor_frame : 0;
+    return TTF_OK;
+}
+
+int ttf_compress_ex(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                    int anchor_mode, int anchor_frame,
+                    void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream) {
+    if (!features || !out_tokens || !out_count || !out_pos_thw) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
+    if (rc == TTF_OK) rc = set_anchor_rule(&p, anchor_mode, anchor_frame);
+    if (rc != TTF_OK) return rc;
+    Scratch s;
+    carve_scratch(p, nullptr, &s);
+    void* ws = nullptr;
+    rc = cached_scratch(s.bytes, (cudaStream_t)stream, &ws);
+    if (rc != TTF_OK) return rc;
+    return compress_impl(p, ws, out_tokens, out_count, out_pos_thw, (cudaStream_t)stream);
+}
+
+int ttf_query_ex(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                 int anchor_mode, int anchor_frame,
+                 int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
+                 int* out_fuse_cnt, ttf_stream_t stream) {
+    if (!features) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
+    if (rc == TTF_OK) rc = set_anchor_rule(&p, anchor_mode, anchor_frame);
     if (rc != TTF_OK) return rc;
     Scratch s;
     carve_scratch(p, nullptr, &s);

@@ -71,7 +71,7 @@ __device__ __forceinline__ int select_in_frame(const unsigned char* __restrict__
         const int c0 = b + lane * 8;
         unsigned bits = 0;
         if (c0 + 8 <= N && ((reinterpret_cast<uintptr_t>(kf + c0) & 7) == 0)) {
-            const uint2 v = *reinterpret_cast<const uint2*>(kf + c0);
+            const uint2 v = __ldcg(reinterpret_cast<const uint2*>(kf + c0));
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 bits |= ((v.x >> (8 * e)) & 0xffu) ? (1u << e) : 0u;
@@ -79,7 +79,7 @@ __device__ __forceinline__ int select_in_frame(const unsigned char* __restrict__
             }
         } else {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) bits |= (c0 + e < N && kf[c0 + e] != 0) ? (1u << e) : 0u;
+            for (int e = 0; e < 8; ++e) bits |= (c0 + e < N && __ldcg(kf + c0 + e) != 0) ? (1u << e) : 0u;
         }
         const int mine = __popc(bits);
         int incl = mine;
@@ -112,7 +112,8 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
     using U = typename CopyUnit<COPY_BYTES>::type;
     const int N = H * W;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    const int a = hdr[HDR_ANCHOR];
+    pdl_wait();                                  // keep flags, dst and survivor counts are complete
+    const int a = __ldcg(hdr + HDR_ANCHOR);
 
     // ---- bookkeeping CTAs: tokens fused into each anchor cell (gather-side, integer, fixed order) --------
     if ((int)blockIdx.x >= ncopy_blocks) {
@@ -126,7 +127,7 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
                 for (int yy = max(0, y - r); yy <= min(H - 1, y + r); ++yy)
                     for (int xx = max(0, x - r); xx <= min(W - 1, x + r); ++xx) {
                         const size_t f = (size_t)k * N + yy * W + xx;
-                        c += (!keep[f] && dst[f] == j) ? 1 : 0;
+                        c += (!__ldcg(keep + f) && __ldcg(dst + f) == j) ? 1 : 0;
                     }
             }
 #pragma unroll
@@ -146,7 +147,7 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
         const int per = (F + kCopyWarps * 32 - 1) / (kCopyWarps * 32);
         const int k0 = tid * per;
         int sum = 0;
-        for (int k = k0; k < min(F, k0 + per); ++k) sum += (k != a) ? cnt[k] : 0;
+        for (int k = k0; k < min(F, k0 + per); ++k) sum += (k != a) ? __ldcg(cnt + k) : 0;
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -158,7 +159,7 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
         int woff = 0;
         for (int ww = 0; ww < w; ++ww) woff += s_warp[ww];
         int run = woff + incl - sum;
-        for (int k = k0; k < min(F, k0 + per); ++k) { s_pre[k] = run; run += (k != a) ? cnt[k] : 0; }
+        for (int k = k0; k < min(F, k0 + per); ++k) { s_pre[k] = run; run += (k != a) ? __ldcg(cnt + k) : 0; }
         if (tid == kCopyWarps * 32 - 1) s_pre[F] = woff + incl;
         __syncthreads();
         pre = s_pre;
@@ -247,16 +248,20 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
     const int grid = ncopy + nfuse;
     const unsigned char* X = reinterpret_cast<const unsigned char*>(p.X);
     unsigned char* out = reinterpret_cast<unsigned char*>(out_tokens);
+    const dim3 g(grid), b(kCopyWarps * 32);
+    // the pre-scanned prefix of very long clips is read through plain loads: order that case by the stream
+    const bool pdl = p.F <= kSmemPrefixMaxF;
     if (vec)
-        k_compact<16><<<grid, kCopyWarps * 32, 0, st>>>(X, row_bytes, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix,
-            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy);
-    else if (esize == 4)
-        k_compact<4><<<grid, kCopyWarps * 32, 0, st>>>(X, row_bytes, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix,
-            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy);
-    else
-        k_compact<2><<<grid, kCopyWarps * 32, 0, st>>>(X, row_bytes, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix,
-            s.keep, s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy);
-    return cudaGetLastError();
+        return launch_pdl_if(pdl, k_compact<16>, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
+                          (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep, (const int*)s.dst,
+                          out, out_pos, out_count, s.fuse_cnt, ncopy);
+    if (esize == 4)
+        return launch_pdl_if(pdl, k_compact<4>, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
+                          (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep, (const int*)s.dst,
+                          out, out_pos, out_count, s.fuse_cnt, ncopy);
+    return launch_pdl_if(pdl, k_compact<2>, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
+                      (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep, (const int*)s.dst,
+                      out, out_pos, out_count, s.fuse_cnt, ncopy);
 }
 
 }  // namespace ttf

@@ -24,24 +24,26 @@ struct Problem {
     int N;              // H * W
     int vec;            // 1 when rows are 16-byte aligned and a multiple of 16 bytes long, else 0
     int lanes_elems;    // channels one lane loads at once: 16 B worth when vec, else 1
-    int nslice;         // channel slices of 32 lanes: ceil(C / (32 * lanes_elems))
+    int cpt;            // norm sweep: chunks of lanes_elems channels per thread per row (1 or 2)
+    int ncb;            // norm sweep: column blocks of 256 * cpt chunks per row
+    int nslice;         // planes of partial squared norms: 8 warps x ncb
+    int nsl;            // anchor pick: channel slices (256 channels when C % 4 == 0, else 32)
     int anchor_mode;    // 0 auto (Eq. auto_anchor), 1 first, 2 last, 3 explicit
     int anchor_arg;     // explicit anchor frame
 };
 
 // Device pointers carved out of one scratch allocation.
 struct Scratch {
-    int* hdr;           // [kHdrInts]  anchor frame, arrival counter of the slices
-    int* done_slice;    // [nslice]    arrival counters of the CTAs of a channel slice (directly after hdr)
+    int* hdr;           // [kHdrInts]  anchor frame, arrival counter of the anchor-pick slices
     int* cnt;           // [F]   preserved tokens per source frame (Eq. gating summed over a frame)
     int* prefix;        // [F+1] exclusive scan of cnt, only used when F > kSmemPrefixMaxF
     float* fcos;        // [F]   cosine of each frame mean to the global mean (Eq. auto_anchor)
     float* Sp;          // [TG, F, C] per-frame channel sums of each token group
     float* S;           // [F, C] per-frame channel sums
-    float* Dp;          // [nslice, F] per-slice share of <S_k, g>
-    float* Qp;          // [nslice, F] per-slice share of |S_k|^2
-    float* Gp;          // [nslice]    per-slice share of |g|^2
-    float* ssq;         // [nslice, F*N] partial squared norms per channel slice
+    float* Dp;          // [nsl, F] per-slice share of <S_k, g>
+    float* Qp;          // [nsl, F] per-slice share of |S_k|^2
+    float* Gp;          // [nsl]    per-slice share of |g|^2
+    float* ssq;         // [nslice, F*N] partial squared norms (one plane per warp and column block)
     float* shat;        // [F*N] best similarity (Eq. argmax)
     int* dst;           // [F*N] best anchor cell (Eq. dst)
     unsigned char* keep;// [F*N] retention mask (Eq. mask)
@@ -64,10 +66,37 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
 
 int sm_count();   // SMs of the current device (cached per device)
 
+// Launch with programmatic dependent launch: the kernel may be scheduled while the previous kernel of the
+// stream drains; it must execute pdl_wait() before it touches anything an earlier kernel wrote, and every
+// kernel launched this way executes pdl_wait() on all paths so that completion stays transitive.
+// Because such a kernel is already alive while its predecessor still writes, whatever the predecessor
+// produces is NOT read-only data for it: it must be read with L2-coherent loads (__ldcg), never through the
+// non-coherent / L1 path that `const __restrict__` pointers and __ldg select.  Only X is truly read-only.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl_if(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st,
+                                 Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {
+    return launch_pdl_if(true, kernel, grid, block, st, args...);
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // device helpers
 // ---------------------------------------------------------------------------------------------------------
 #ifdef __CUDACC__
+
+// griddepcontrol: wait = all kernels this one depends on have completed and their writes are visible (a no-op
+// for a normally launched kernel); launch_dependents = the next kernel of the stream may be scheduled.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 struct bf16_t { uint16_t bits; };   // storage type only: all arithmetic is on the widened fp32 value
 
@@ -120,7 +149,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // 1 / max(||x||, floor) from the per-slice partial squared norms of token f, summed in slice order
 __device__ __forceinline__ float inv_norm(const float* __restrict__ ssq, int nslice, size_t FN, size_t f) {
     float s = 0.f;
-    for (int q = 0; q < nslice; ++q) s += ssq[(size_t)q * FN + f];
+    for (int q = 0; q < nslice; ++q) s += __ldcg(ssq + (size_t)q * FN + f);
     return 1.0f / fmaxf(sqrtf(s), kNormFloor);
 }
 

@@ -23,11 +23,13 @@ k_match_generic(const T* __restrict__ X, int F, int H, int W, int C, int r, floa
                 float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep,
                 int* __restrict__ cnt)
 {
+    pdl_launch_dependents();
+    pdl_wait();                                  // norms and the anchor index are complete
     const int N = H * W;
     const int i = blockIdx.x % N;
     const int chunk = blockIdx.x / N;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int a = hdr[HDR_ANCHOR];
+    const int a = __ldcg(hdr + HDR_ANCHOR);
     const int y = i / W, x = i - y * W;
     const size_t FN = (size_t)F * N;
     const int y_lo = max(0, y - r), y_hi = min(H - 1, y + r);
@@ -155,7 +157,9 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
     const int k0 = (blockIdx.x / N) * FR;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int g = lane >> 2, tig = lane & 3;
-    const int a = hdr[HDR_ANCHOR];
+    pdl_launch_dependents();
+    pdl_wait();                                  // norms and the anchor index are complete
+    const int a = __ldcg(hdr + HDR_ANCHOR);
     const int y = i / W, x = i - y * W;
     const int side = 2 * r + 1, ncand = side * side;
     const size_t FN = (size_t)F * N;
@@ -264,10 +268,9 @@ template <int MT, int NT>
 static cudaError_t launch_mma_t(const Problem& p, const Scratch& s, float* shat, int* dst, unsigned char* keep,
                                 cudaStream_t st) {
     const long long chunks = (p.F + 16 * MT - 1) / (16 * MT);
-    k_match_mma<MT, NT><<<(unsigned)(chunks * p.N), kMmaWarps * 32, 0, st>>>(
-        reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t, p.nslice, s.hdr, s.ssq, shat, dst,
-        keep, s.cnt);
-    return cudaGetLastError();
+    return launch_pdl(k_match_mma<MT, NT>, dim3((unsigned)(chunks * p.N)), dim3(kMmaWarps * 32), st,
+                      reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t, p.nslice,
+                      (const int*)s.hdr, (const float*)s.ssq, shat, dst, keep, s.cnt);
 }
 
 template <typename T, int V>
@@ -282,10 +285,9 @@ static cudaError_t launch_generic_t(const Problem& p, const Scratch& s, float* s
         if (fchunk < kMatchWarps) fchunk = kMatchWarps;
     }
     const long long nchunk = (p.F + fchunk - 1) / fchunk;
-    k_match_generic<T, V><<<(unsigned)(nchunk * p.N), kMatchWarps * 32, 0, st>>>(
-        reinterpret_cast<const T*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t, fchunk, p.nslice, s.hdr, s.ssq,
-        shat, dst, keep, s.cnt);
-    return cudaGetLastError();
+    return launch_pdl(k_match_generic<T, V>, dim3((unsigned)(nchunk * p.N)), dim3(kMatchWarps * 32), st,
+                      reinterpret_cast<const T*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t, fchunk, p.nslice,
+                      (const int*)s.hdr, (const float*)s.ssq, shat, dst, keep, s.cnt);
 }
 
 cudaError_t launch_match(const Problem& p, const Scratch& s, float* shat, int* dst, unsigned char* keep,

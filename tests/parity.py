@@ -37,21 +37,25 @@ def to_bits(t: torch.Tensor) -> np.ndarray:
 
 
 def check_clip(X: np.ndarray, r: int, t: float, *, stream=None, workspace=None, oracle=None,
-               require_anchor=True) -> dict:
+               require_anchor=True, anchor_mode: int = 0, anchor_frame: int = 0) -> dict:
     """Runs ttf_query and ttf_compress on X and compares with the oracle.  Returns a small report."""
     F, H, W, C = X.shape
     N = H * W
-    R = oracle if oracle is not None else O.compress(X, r, t)
+    fixed = {0: None, 1: 0, 2: F - 1, 3: anchor_frame}[anchor_mode]       # first / last / explicit anchors
+    R = oracle if oracle is not None else O.compress(X, r, t, anchor_frame=fixed)
     Xd = to_device(X)
 
-    q = P.ttf_query(Xd, r, t, stream=stream, workspace=workspace)
-    toks, cnt, pos = P.ttf_compress(Xd, r, t, stream=stream, workspace=workspace)
+    kw = dict(stream=stream, workspace=workspace, anchor_mode=anchor_mode, anchor_frame=anchor_frame)
+    q = P.ttf_query(Xd, r, t, **kw)
+    toks, cnt, pos = P.ttf_compress(Xd, r, t, **kw)
     torch.cuda.synchronize()
 
     a_gpu = int(q["anchor"].item())
     cos_sorted = np.sort(R.anchor_cos)
     margin = float(cos_sorted[-1] - cos_sorted[-2]) if F > 1 else float("inf")
-    if a_gpu != R.anchor:
+    if fixed is not None:
+        assert a_gpu == fixed, f"anchor {a_gpu} != requested {fixed}"
+    elif a_gpu != R.anchor:
         assert not require_anchor or margin < ANCHOR_MARGIN, f"anchor {a_gpu} != oracle {R.anchor} (margin {margin:.3g})"
         R = O.compress(X, r, t, anchor_frame=a_gpu)
 

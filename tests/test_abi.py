@@ -64,6 +64,9 @@ def test_null_and_nonfinite_arguments_are_rejected_before_any_launch(lib):
     assert lib.ttf_compress_ws(fake, 4, 4, 4, 8, 1, 0.7, 0, fake, fake, fake, ctypes.c_void_p(4096 + 8), 1 << 30, None) == 3
     assert lib.ttf_query(None, 4, 4, 4, 8, 1, 0.7, 0, None, None, None, None, None, None) == 1
     assert lib.ttf_compress_host(None, 4, 4, 4, 8, 1, 0.7, 0, fake, fake, fake) == 1
+    assert lib.ttf_compress_ex(fake, 4, 4, 4, 8, 1, 0.7, 0, 4, 0, fake, fake, fake, None) == 1      # unknown rule
+    assert lib.ttf_compress_ex(fake, 4, 4, 4, 8, 1, 0.7, 0, 3, 4, fake, fake, fake, None) == 1      # frame >= F
+    assert lib.ttf_query_ex(fake, 4, 4, 4, 8, 1, 0.7, 0, 3, -1, None, None, None, None, None, None) == 1
 
 
 def test_decode_alignment_helper():

@@ -64,6 +64,17 @@ def test_identical_frames_and_zero_tokens():
     check_clip(np.zeros((3, 3, 3, 16), np.float32), 1, 0.5)
 
 
+@pytest.mark.parametrize("mode,frame", [(1, 0), (2, 0), (3, 0), (3, 2), (3, 4)])
+def test_fixed_anchor_rules(mode, frame):
+    """first / last / explicit anchors (the paper's Table 1 variants)"""
+    for dtype, shape in (("bf16", (5, 6, 7, 256)), ("f32", (5, 4, 5, 40))):
+        X = corr_clip(*shape, seed=21 + mode + frame, dtype=dtype)
+        rep = check_clip(X, 1, 0.7, anchor_mode=mode, anchor_frame=frame)
+        assert rep["anchor"] == {1: 0, 2: shape[0] - 1, 3: frame}[mode]
+    with pytest.raises(P.TTFError):
+        P.ttf_query(to_device(X), 1, 0.7, anchor_mode=3, anchor_frame=5)
+
+
 def test_misaligned_base_pointer_takes_scalar_path():
     F, H, W, C = 3, 4, 5, 64
     X = corr_clip(F, H, W, C, seed=12, dtype="bf16")
