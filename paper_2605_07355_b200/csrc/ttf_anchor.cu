@@ -9,7 +9,7 @@
 // is reduced over the warp with a shuffle fold and stored as one partial per (warp, token); consumers add the
 // partials in a fixed order.
 //
-// k_anchor_pick.  One CTA per 256-channel slice adds the token-group partials into S[:, slice], forms
+// k_anchor_pick.  One CTA per 64-channel slice adds the token-group partials into S_k[slice] (registers), forms
 // g[slice] = sum_k S_k[slice] and the slice's shares of <S_k, g>, |S_k|^2, |g|^2.  The slices count
 // themselves; the last one adds the shares in slice order, takes the cosines (the factors 1/N and 1/(FN) of
 // Eq. auto_anchor cancel in a cosine) and the arg max (lowest frame on ties) and resets the counter.  Which
@@ -144,11 +144,11 @@ static cudaError_t launch_sum_t(const Problem& p, const Scratch& s, cudaStream_t
 }
 
 // ---------------------------------------------------------------------------------------------------------
-constexpr int kPickFB = 4;           // frames per warp in flight
+constexpr int kPickFB = 4;           // frames per thread held in registers
+constexpr int kPickLanes = 16;       // threads across a slice (each V channels); 16 frame rows per CTA
 
 struct PickArgs {
     const float* Sp;    // [TG, F, C]
-    float* S;           // [F, C]
     float* Dp;          // [nsl, F] slice shares of <S_k, g>
     float* Qp;          // [nsl, F] slice shares of |S_k|^2
     float* Gp;          // [nsl]    slice shares of |g|^2
@@ -159,13 +159,14 @@ struct PickArgs {
 };
 
 template <int V> __device__ __forceinline__ void load_f32(const float* p, float (&x)[V]);
-template <> __device__ __forceinline__ void load_f32<8>(const float* p, float (&x)[8]) {
-    const float4 a = __ldcg(reinterpret_cast<const float4*>(p)), b = __ldcg(reinterpret_cast<const float4*>(p) + 1);
-    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+template <> __device__ __forceinline__ void load_f32<4>(const float* p, float (&x)[4]) {
+    const float4 a = __ldcg(reinterpret_cast<const float4*>(p));
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w;
 }
 template <> __device__ __forceinline__ void load_f32<1>(const float* p, float (&x)[1]) { x[0] = __ldcg(p); }
 
-// V channels per lane: 8 when C is a multiple of 4 (16-byte loads of fp32), else 1
+// A CTA owns a slice of 16*V channels: thread = (frame row 0..15, lane 0..15 with V channels).
+// V = 4 when C is a multiple of 4 (16-byte loads of the fp32 partial sums), else 1.
 template <int V>
 __global__ void __launch_bounds__(kNormThreads)
 k_anchor_pick(int F, int C, int TG, int nsl, PickArgs A)
@@ -173,8 +174,8 @@ k_anchor_pick(int F, int C, int TG, int nsl, PickArgs A)
     pdl_launch_dependents();
     const int q = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    __shared__ float sm[kNormWarps][32 * V];
-    __shared__ float s_g[32 * V];
+    const int cl = tid & (kPickLanes - 1), row = tid / kPickLanes;
+    __shared__ float s_gp[kNormThreads / kPickLanes][kPickLanes * V];
     __shared__ float s_red[kNormWarps];
     __shared__ int s_redi[kNormWarps];
     __shared__ int s_flag;
@@ -189,96 +190,80 @@ k_anchor_pick(int F, int C, int TG, int nsl, PickArgs A)
         return;
     }
 
-    // warp w owns frames w, w+8, ...; lane owns V channels of the slice; kPickFB frames per warp in flight
-    const int c0 = (q * 32 + lane) * V;
-    bool active;
-    if constexpr (V == 8) active = c0 < C;           // C % 4 == 0: a lane's 8 channels may be cut to 4
-    else active = c0 < C;
-    const bool half = (V == 8) && active && (c0 + 4 >= C);   // only the first float4 is inside the row
-    auto ld = [&](const float* p, float (&x)[V]) {
-        if constexpr (V == 8) {
-            if (half) {
-                const float4 a = __ldcg(reinterpret_cast<const float4*>(p));
-                x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = x[5] = x[6] = x[7] = 0.f;
-            } else load_f32<8>(p, x);
-        } else load_f32<1>(p, x);
-    };
-    auto st = [&](float* p, const float (&x)[V]) {
-        if constexpr (V == 8) {
-            reinterpret_cast<float4*>(p)[0] = make_float4(x[0], x[1], x[2], x[3]);
-            if (!half) reinterpret_cast<float4*>(p)[1] = make_float4(x[4], x[5], x[6], x[7]);
-        } else p[0] = x[0];
-    };
+    const int c0 = (q * kPickLanes + cl) * V;
+    const bool active = c0 < C;                      // C % V == 0
+    constexpr int kRows = kNormThreads / kPickLanes; // 16
+    const bool resident = F <= kRows * kPickFB;      // all frame sums of this thread stay in registers
 
-    float gacc[V];
-#pragma unroll
-    for (int v = 0; v < V; ++v) gacc[v] = 0.f;
-    for (int kb = w; kb < F; kb += kNormWarps * kPickFB) {
-        float acc[kPickFB][V];
+    // S_k[c] = sum over token groups (ascending), for the frames row, row+16, ... of this thread
+    auto frame_sums = [&](int kb, float (&acc)[kPickFB][V]) {
 #pragma unroll
         for (int jj = 0; jj < kPickFB; ++jj)
 #pragma unroll
             for (int v = 0; v < V; ++v) acc[jj][v] = 0.f;
+#pragma unroll 4
         for (int t2 = 0; t2 < TG; ++t2) {
 #pragma unroll
             for (int jj = 0; jj < kPickFB; ++jj) {
-                const int kk = kb + jj * kNormWarps;
+                const int kk = kb + jj * kRows;
                 if (active && kk < F) {
                     float x[V];
-                    ld(A.Sp + ((size_t)t2 * F + kk) * C + c0, x);
+                    load_f32<V>(A.Sp + ((size_t)t2 * F + kk) * C + c0, x);
 #pragma unroll
                     for (int v = 0; v < V; ++v) acc[jj][v] += x[v];
                 }
             }
         }
+    };
+
+    float acc[kPickFB][V];
+    float gacc[V];
 #pragma unroll
-        for (int jj = 0; jj < kPickFB; ++jj) {
-            const int kk = kb + jj * kNormWarps;
-            if (active && kk < F) {
-                st(A.S + (size_t)kk * C + c0, acc[jj]);
+    for (int v = 0; v < V; ++v) gacc[v] = 0.f;
+    // trip counts are the same for every thread (the shuffles below need whole warps); frames past F add zeros
+    for (int kb0 = 0; kb0 < F; kb0 += kRows * kPickFB) {
+        const int kb = kb0 + row;
+        frame_sums(kb, acc);
 #pragma unroll
-                for (int v = 0; v < V; ++v) gacc[v] += acc[jj][v];
-            }
-        }
+        for (int jj = 0; jj < kPickFB; ++jj)
+#pragma unroll
+            for (int v = 0; v < V; ++v) gacc[v] += acc[jj][v];      // frames past F contributed zeros
     }
 #pragma unroll
-    for (int v = 0; v < V; ++v) sm[w][lane * V + v] = gacc[v];
+    for (int v = 0; v < V; ++v) s_gp[row][cl * V + v] = gacc[v];
     __syncthreads();
-    for (int idx = tid; idx < 32 * V; idx += kNormThreads) {
+    float gl[V];                                     // g[c] = sum_k S_k[c], rows combined in row order
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
         float g = 0.f;
 #pragma unroll
-        for (int ww = 0; ww < kNormWarps; ++ww) g += sm[ww][idx];
-        s_g[idx] = g;                                // channels past C hold 0
+        for (int rr = 0; rr < kRows; ++rr) g += s_gp[rr][cl * V + v];
+        gl[v] = g;
     }
-    __syncthreads();
-    float gl[V];
-#pragma unroll
-    for (int v = 0; v < V; ++v) gl[v] = s_g[lane * V + v];
-    for (int kb = w; kb < F; kb += kNormWarps * kPickFB) {
-        float d[kPickFB], qq[kPickFB];
+    for (int kb0 = 0; kb0 < F; kb0 += kRows * kPickFB) {
+        const int kb = kb0 + row;
+        if (!resident) frame_sums(kb, acc);
 #pragma unroll
         for (int jj = 0; jj < kPickFB; ++jj) {
-            const int kk = kb + jj * kNormWarps;
-            d[jj] = 0.f; qq[jj] = 0.f;
-            if (active && kk < F) {
-                float x[V];
-                ld(A.S + (size_t)kk * C + c0, x);    // written above by this very thread
+            const int kk = kb + jj * kRows;
+            float d = 0.f, qq = 0.f;
 #pragma unroll
-                for (int v = 0; v < V; ++v) { d[jj] = fmaf(x[v], gl[v], d[jj]); qq[jj] = fmaf(x[v], x[v], qq[jj]); }
+            for (int v = 0; v < V; ++v) { d = fmaf(acc[jj][v], gl[v], d); qq = fmaf(acc[jj][v], acc[jj][v], qq); }
+#pragma unroll
+            for (int o = kPickLanes / 2; o > 0; o >>= 1) {
+                d += __shfl_xor_sync(0xffffffffu, d, o);
+                qq += __shfl_xor_sync(0xffffffffu, qq, o);
             }
-        }
-#pragma unroll
-        for (int jj = 0; jj < kPickFB; ++jj) {
-            const int kk = kb + jj * kNormWarps;
-            const float ds = warp_sum(d[jj]), qs = warp_sum(qq[jj]);
-            if (lane == 0 && kk < F) { A.Dp[(size_t)q * F + kk] = ds; A.Qp[(size_t)q * F + kk] = qs; }
+            if (cl == 0 && kk < F) { A.Dp[(size_t)q * F + kk] = d; A.Qp[(size_t)q * F + kk] = qq; }
         }
     }
     if (w == 0) {
         float gg = 0.f;
+        if (row == 0) {
 #pragma unroll
-        for (int v = 0; v < V; ++v) gg = fmaf(gl[v], gl[v], gg);
-        gg = warp_sum(gg);
+            for (int v = 0; v < V; ++v) gg = fmaf(gl[v], gl[v], gg);
+        }
+        gg = warp_sum(gg);                           // lanes 16..31 (row 1) add zeros
         if (lane == 0) A.Gp[q] = gg;
     }
 
@@ -349,12 +334,12 @@ cudaError_t launch_norm_anchor(const Problem& p, const Scratch& s, int* out_anch
     else e = p.vec ? launch_sum_t<bf16_t, 8>(p, s, st) : launch_sum_t<bf16_t, 1>(p, s, st);
     if (e != cudaSuccess) return e;
     PickArgs A;
-    A.Sp = s.Sp; A.S = s.S; A.Dp = s.Dp; A.Qp = s.Qp; A.Gp = s.Gp; A.fcos = s.fcos; A.hdr = s.hdr;
+    A.Sp = s.Sp; A.Dp = s.Dp; A.Qp = s.Qp; A.Gp = s.Gp; A.fcos = s.fcos; A.hdr = s.hdr;
     A.out_anchor = out_anchor; A.mode = p.anchor_mode; A.arg = p.anchor_arg;
     const int TG = norm_token_groups(p);
     const bool fixed = p.anchor_mode != 0;
     if (p.C % 4 == 0)
-        return launch_pdl(k_anchor_pick<8>, dim3(fixed ? 1 : p.nsl), dim3(kNormThreads), st, p.F, p.C, TG, p.nsl, A);
+        return launch_pdl(k_anchor_pick<4>, dim3(fixed ? 1 : p.nsl), dim3(kNormThreads), st, p.F, p.C, TG, p.nsl, A);
     return launch_pdl(k_anchor_pick<1>, dim3(fixed ? 1 : p.nsl), dim3(kNormThreads), st, p.F, p.C, TG, p.nsl, A);
 }
 

@@ -66,7 +66,6 @@ void carve_scratch(const Problem& p, void* base, Scratch* s) {
     s->prefix = (int*)take(sizeof(int) * ((size_t)p.F + 1));
     s->fcos = (float*)take(sizeof(float) * p.F);
     s->Sp = (float*)take(sizeof(float) * (size_t)norm_token_groups(p) * p.F * p.C);
-    s->S = (float*)take(sizeof(float) * (size_t)p.F * p.C);
     s->Dp = (float*)take(sizeof(float) * (size_t)p.nsl * p.F);
     s->Qp = (float*)take(sizeof(float) * (size_t)p.nsl * p.F);
     s->Gp = (float*)take(sizeof(float) * (size_t)p.nsl);
@@ -97,7 +96,7 @@ static int make_problem(const void* X, int F, int H, int W, int C, int r, float 
     p->cpt = chunks <= 256 ? 1 : 2;
     p->ncb = (int)((chunks + 256LL * p->cpt - 1) / (256LL * p->cpt));
     p->nslice = 8 * p->ncb;
-    p->nsl = C % 4 == 0 ? (C + 255) / 256 : (C + 31) / 32;
+    p->nsl = C % 4 == 0 ? (C + 63) / 64 : (C + 15) / 16;
     p->anchor_mode = 0; p->anchor_arg = 0;
     return TTF_OK;
 }

@@ -27,7 +27,7 @@ struct Problem {
     int cpt;            // norm sweep: chunks of lanes_elems channels per thread per row (1 or 2)
     int ncb;            // norm sweep: column blocks of 256 * cpt chunks per row
     int nslice;         // planes of partial squared norms: 8 warps x ncb
-    int nsl;            // anchor pick: channel slices (256 channels when C % 4 == 0, else 32)
+    int nsl;            // anchor pick: channel slices (64 channels when C % 4 == 0, else 16)
     int anchor_mode;    // 0 auto (Eq. auto_anchor), 1 first, 2 last, 3 explicit
     int anchor_arg;     // explicit anchor frame
 };
@@ -39,7 +39,6 @@ struct Scratch {
     int* prefix;        // [F+1] exclusive scan of cnt, only used when F > kSmemPrefixMaxF
     float* fcos;        // [F]   cosine of each frame mean to the global mean (Eq. auto_anchor)
     float* Sp;          // [TG, F, C] per-frame channel sums of each token group
-    float* S;           // [F, C] per-frame channel sums
     float* Dp;          // [nsl, F] per-slice share of <S_k, g>
     float* Qp;          // [nsl, F] per-slice share of |S_k|^2
     float* Gp;          // [nsl]    per-slice share of |g|^2
