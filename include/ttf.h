@@ -170,7 +170,7 @@ int ttf_query_static(const void* features, int F, int H, int W, int C, int r, fl
  * on its own stream.  ttf_profile_end waits for those events and returns, per kernel kind, the summed
  * device time in milliseconds and the number of launches; `kinds` is the length of both arrays
  * (TTF_KERNEL_KINDS covers all).  Kinds: 0 norm + frame-sum sweep with the anchor pick, 1 windowed match +
- * gate, 2 compaction gather (with the frame-count prefix of clips longer than 2048 frames), 3 fuse-count
+ * gate, 2 compaction gather (with the frame-count prefix of clips longer than 1024 frames), 3 fuse-count
  * bookkeeping of ttf_query.  Profiling is process-wide and meant for benchmarks; leave it off otherwise.
  */
 #define TTF_KERNEL_KINDS 4

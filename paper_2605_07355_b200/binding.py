@@ -13,7 +13,7 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libttf_b200.so")
+LIB_PATH = os.environ.get("TTF_B200_LIB") or os.path.join(_HERE, "libttf_b200.so")
 
 TTF_DTYPE_F32, TTF_DTYPE_BF16 = 0, 1
 TTF_OK = 0

@@ -9,7 +9,7 @@
 // is reduced over the warp with a shuffle fold and stored as one partial per (warp, token); consumers add the
 // partials in a fixed order.
 //
-// k_anchor_pick.  One CTA per 64-channel slice adds the token-group partials into S_k[slice] (registers), forms
+// k_anchor_pick.  One CTA per 32-channel slice adds the token-group partials into S_k[slice] (registers), forms
 // g[slice] = sum_k S_k[slice] and the slice's shares of <S_k, g>, |S_k|^2, |g|^2.  The slices count
 // themselves; the last one adds the shares in slice order, takes the cosines (the factors 1/N and 1/(FN) of
 // Eq. auto_anchor cancel in a cosine) and the arg max (lowest frame on ties) and resets the counter.  Which
@@ -20,11 +20,19 @@ namespace ttf {
 
 constexpr int kNormWarps = 8;
 constexpr int kNormThreads = kNormWarps * 32;
-constexpr int kRowBatch = 4;         // rows in flight per step (times two with the prefetch)
+constexpr int kMaxTG = 16;           // token groups per frame (partial frame sums kept per group)
+#ifndef TTF_ROWBATCH
+#define TTF_ROWBATCH 4
+#endif
+#ifndef TTF_NORM_MINBLOCKS
+#define TTF_NORM_MINBLOCKS 2
+#endif
+constexpr int kRowBatch = TTF_ROWBATCH;   // rows in flight per step (times two with the prefetch): 2 or 4
 
 // Sum of v[u] over the warp for u = 0..3 with 6 shuffles; lanes with (lane & 7) == 0 hold the total of token
 // u = 2*bit4 + bit3 of their lane index.
-__device__ __forceinline__ float fold4(float (&v)[4], int lane) {
+template <int NV> __device__ __forceinline__ float fold4(float (&v)[NV], int lane) {
+    static_assert(NV >= 4, "fold4 needs four values");
     {
         const bool up = lane & 16;
 #pragma unroll
@@ -58,12 +66,16 @@ template <int V> __device__ __forceinline__ void store_f32(float* p, const float
 
 // CPT: 16-byte chunks per thread per row (column blocks of 256*CPT chunks are walked one after the other)
 template <typename T, int V, int CPT>
-__global__ void __launch_bounds__(kNormThreads)
+__global__ void __launch_bounds__(kNormThreads, TTF_NORM_MINBLOCKS)
 k_norm_sum(const T* __restrict__ X, int F, int N, int C, int TG, int ncb,
-           float* __restrict__ Sp, float* __restrict__ ssq, int* __restrict__ cnt)
+           float* __restrict__ Sp, float* __restrict__ ssq, int* __restrict__ cnt, int* __restrict__ hdr)
 {
     using L = Loader<T, V>;
     pdl_launch_dependents();
+    // This kernel may be scheduled while the previous call's gather still runs (it shares the scratch) or
+    // while an upstream kernel still writes X: nothing is read or written before the wait.
+    pdl_wait();
+    trace_mark(hdr, 0, false);
     const int k = blockIdx.x / TG, tg = blockIdx.x - k * TG;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const size_t FN = (size_t)F * N;
@@ -90,7 +102,7 @@ k_norm_sum(const T* __restrict__ X, int F, int N, int C, int TG, int ncb,
             for (int u = 0; u < kRowBatch; ++u)
 #pragma unroll
                 for (int j = 0; j < CPT; ++j)
-                    d[u][j] = (on[j] && i0 + u < i_end) ? L::load_raw(frame + (size_t)(i0 + u) * C + c0[j]) : L::zero();
+                    d[u][j] = (on[j] && i0 + u < i_end) ? L::load_raw_cg(frame + (size_t)(i0 + u) * C + c0[j]) : L::zero();
         };
         if (i_begin < i_end) load_batch(cur, i_begin);
         for (int i0 = i_begin; i0 < i_end; i0 += kRowBatch) {
@@ -108,9 +120,19 @@ k_norm_sum(const T* __restrict__ X, int F, int N, int C, int TG, int ncb,
                 }
                 ss[u] = s;
             }
-            const float tot = fold4(ss, lane);
-            const int u = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
-            if ((lane & 7) == 0 && i0 + u < i_end) ssq[(size_t)(cb * kNormWarps + w) * FN + (size_t)k * N + i0 + u] = tot;
+            float tot;
+            int u;
+            if constexpr (kRowBatch == 4) {
+                tot = fold4<kRowBatch>(ss, lane);
+                u = ((lane >> 4) & 1) * 2 + ((lane >> 3) & 1);
+            } else {
+                const bool up = lane & 16;
+                tot = (up ? ss[1] : ss[0]) + __shfl_xor_sync(0xffffffffu, up ? ss[0] : ss[1], 16);
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) tot += __shfl_xor_sync(0xffffffffu, tot, o);
+                u = (lane >> 4) & 1;
+            }
+            if ((lane & (kRowBatch == 4 ? 7 : 15)) == 0 && i0 + u < i_end) ssq[(size_t)(cb * kNormWarps + w) * FN + (size_t)k * N + i0 + u] = tot;
 #pragma unroll
             for (int uu = 0; uu < kRowBatch; ++uu)
 #pragma unroll
@@ -121,14 +143,17 @@ k_norm_sum(const T* __restrict__ X, int F, int N, int C, int TG, int ncb,
             if (on[j]) store_f32<V>(Sp + ((size_t)tg * F + k) * C + c0[j], col[j]);
     }
     if (tg == 0 && tid == 0) cnt[k] = 0;            // survivor counters start at zero for the matching kernel
+    trace_mark(hdr, 0, true);
 }
 
 int norm_token_groups(const Problem& p) {
-    // shape-only rule (the order of every sum must not depend on the device): about 200 CTAs or more, at
-    // least 8 rows per CTA
-    int tg = 1;
-    while (tg < 64 && (long long)p.F * tg < 192 && p.N / (tg * 2) >= 8) tg *= 2;
-    return tg;
+    // shape-only rule (the order of every sum must not depend on the device): F * TG close to, and not above,
+    // 296 CTAs (two per SM on a 148-SM part), at least 8 rows per CTA, at most kMaxTG groups
+    long long tg = 296 / p.F;
+    if (tg > p.N / 8) tg = p.N / 8;
+    if (tg > kMaxTG) tg = kMaxTG;
+    if (tg < 1) tg = 1;
+    return (int)tg;
 }
 
 template <typename T, int V>
@@ -137,15 +162,15 @@ static cudaError_t launch_sum_t(const Problem& p, const Scratch& s, cudaStream_t
     const unsigned blocks = (unsigned)((long long)p.F * TG);
     const T* X = reinterpret_cast<const T*>(p.X);
     if (p.cpt == 1)
-        k_norm_sum<T, V, 1><<<blocks, kNormThreads, 0, st>>>(X, p.F, p.N, p.C, TG, p.ncb, s.Sp, s.ssq, s.cnt);
-    else
-        k_norm_sum<T, V, 2><<<blocks, kNormThreads, 0, st>>>(X, p.F, p.N, p.C, TG, p.ncb, s.Sp, s.ssq, s.cnt);
-    return cudaGetLastError();
+        return launch_pdl(k_norm_sum<T, V, 1>, dim3(blocks), dim3(kNormThreads), st, X, p.F, p.N, p.C, TG, p.ncb,
+                          s.Sp, s.ssq, s.cnt, s.hdr);
+    return launch_pdl(k_norm_sum<T, V, 2>, dim3(blocks), dim3(kNormThreads), st, X, p.F, p.N, p.C, TG, p.ncb,
+                      s.Sp, s.ssq, s.cnt, s.hdr);
 }
 
 // ---------------------------------------------------------------------------------------------------------
-constexpr int kPickFB = 4;           // frames per thread held in registers
-constexpr int kPickLanes = 16;       // threads across a slice (each V channels); 16 frame rows per CTA
+constexpr int kPickFB = 2;           // frames per thread held in registers
+constexpr int kPickLanes = 8;        // threads across a slice (each V channels); 32 frame rows per CTA
 
 struct PickArgs {
     const float* Sp;    // [TG, F, C]
@@ -165,7 +190,7 @@ template <> __device__ __forceinline__ void load_f32<4>(const float* p, float (&
 }
 template <> __device__ __forceinline__ void load_f32<1>(const float* p, float (&x)[1]) { x[0] = __ldcg(p); }
 
-// A CTA owns a slice of 16*V channels: thread = (frame row 0..15, lane 0..15 with V channels).
+// A CTA owns a slice of 8*V channels: thread = (frame row 0..31, lane 0..7 with V channels).
 // V = 4 when C is a multiple of 4 (16-byte loads of the fp32 partial sums), else 1.
 template <int V>
 __global__ void __launch_bounds__(kNormThreads)
@@ -180,7 +205,9 @@ k_anchor_pick(int F, int C, int TG, int nsl, PickArgs A)
     __shared__ int s_redi[kNormWarps];
     __shared__ int s_flag;
 
+    trace_mark(A.hdr, 1, false);
     pdl_wait();                                      // the sweep's partial sums are complete and visible
+    trace_mark(A.hdr, 4, false);
     if (A.mode != 0) {                               // fixed anchors of Table 1 (first / last) or an explicit frame
         if (q == 0 && tid == 0) {
             const int a = A.mode == 1 ? 0 : (A.mode == 2 ? F - 1 : A.arg);
@@ -192,7 +219,7 @@ k_anchor_pick(int F, int C, int TG, int nsl, PickArgs A)
 
     const int c0 = (q * kPickLanes + cl) * V;
     const bool active = c0 < C;                      // C % V == 0
-    constexpr int kRows = kNormThreads / kPickLanes; // 16
+    constexpr int kRows = kNormThreads / kPickLanes; // 32
     const bool resident = F <= kRows * kPickFB;      // all frame sums of this thread stay in registers
 
     // S_k[c] = sum over token groups (ascending), for the frames row, row+16, ... of this thread
@@ -201,12 +228,12 @@ k_anchor_pick(int F, int C, int TG, int nsl, PickArgs A)
         for (int jj = 0; jj < kPickFB; ++jj)
 #pragma unroll
             for (int v = 0; v < V; ++v) acc[jj][v] = 0.f;
-#pragma unroll 4
-        for (int t2 = 0; t2 < TG; ++t2) {
+#pragma unroll
+        for (int t2 = 0; t2 < kMaxTG; ++t2) {       // all loads of the batch are independent and issued together
 #pragma unroll
             for (int jj = 0; jj < kPickFB; ++jj) {
                 const int kk = kb + jj * kRows;
-                if (active && kk < F) {
+                if (active && kk < F && t2 < TG) {
                     float x[V];
                     load_f32<V>(A.Sp + ((size_t)t2 * F + kk) * C + c0, x);
 #pragma unroll
@@ -263,7 +290,7 @@ k_anchor_pick(int F, int C, int TG, int nsl, PickArgs A)
 #pragma unroll
             for (int v = 0; v < V; ++v) gg = fmaf(gl[v], gl[v], gg);
         }
-        gg = warp_sum(gg);                           // lanes 16..31 (row 1) add zeros
+        gg = warp_sum(gg);                           // the lanes of rows 1..3 add zeros
         if (lane == 0) A.Gp[q] = gg;
     }
 
@@ -272,6 +299,7 @@ k_anchor_pick(int F, int C, int TG, int nsl, PickArgs A)
     __syncthreads();
     if (tid == 0) s_flag = (atomicAdd(&A.hdr[HDR_DONE_ALL], 1) == nsl - 1);
     __syncthreads();
+    trace_mark(A.hdr, 4, true);
     if (!s_flag) return;
     __threadfence();
 
@@ -290,11 +318,13 @@ k_anchor_pick(int F, int C, int TG, int nsl, PickArgs A)
     for (int kb = 0; kb < F; kb += kNormThreads / 8) {
         const int kk = kb + (tid >> 3), part = tid & 7;
         float d = 0.f, s2 = 0.f;
-        if (kk < F)
+        if (kk < F) {
+#pragma unroll 16
             for (int qq = part; qq < nsl; qq += 8) {
                 d += __ldcg(A.Dp + (size_t)qq * F + kk);
                 s2 += __ldcg(A.Qp + (size_t)qq * F + kk);
             }
+        }
 #pragma unroll
         for (int o = 1; o < 8; o <<= 1) {
             d += __shfl_xor_sync(0xffffffffu, d, o);
@@ -326,6 +356,7 @@ k_anchor_pick(int F, int C, int TG, int nsl, PickArgs A)
         if (A.out_anchor) *A.out_anchor = bi;
         A.hdr[HDR_DONE_ALL] = 0;                     // ready for the next call
     }
+    trace_mark(A.hdr, 1, true);
 }
 
 cudaError_t launch_norm_anchor(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st) {

@@ -96,7 +96,7 @@ static int make_problem(const void* X, int F, int H, int W, int C, int r, float 
     p->cpt = chunks <= 256 ? 1 : 2;
     p->ncb = (int)((chunks + 256LL * p->cpt - 1) / (256LL * p->cpt));
     p->nslice = 8 * p->ncb;
-    p->nsl = C % 4 == 0 ? (C + 63) / 64 : (C + 15) / 16;
+    p->nsl = C % 4 == 0 ? (C + 31) / 32 : (C + 7) / 8;
     p->anchor_mode = 0; p->anchor_arg = 0;
     return TTF_OK;
 }

@@ -3,11 +3,11 @@
 //
 // The output position of a preserved source token is N plus the number of preserved source tokens before it
 // in flat (k, i) order.  That exclusive prefix is taken in two levels: the per-frame survivor counts written
-// by the matching kernel are scanned by every CTA (shared memory, or a pre-scanned array for very long
+// by the matching kernel are scanned by every warp for itself (shuffles; a pre-scanned array for very long
 // clips), and inside a frame the rank is a population count over the frame's keep flags.  The gather is then
-// driven from the OUTPUT side: every CTA owns an equal, contiguous range of output rows, finds their source
-// rows by rank/select and copies them, so the bytes per CTA are the same no matter how unevenly the
-// survivors are spread over the frames.  No CTA ever waits for another one.
+// driven from the OUTPUT side: one warp per output row finds the source row by rank/select and copies it
+// with all of its 16-byte loads in flight at once, so the work per warp is the same no matter how unevenly
+// the survivors are spread over the frames.  No warp ever waits for another one.
 #include "ttf_internal.cuh"
 
 namespace ttf {
@@ -61,8 +61,11 @@ template <> struct CopyUnit<16> { using type = uint4; };
 template <> struct CopyUnit<4> { using type = uint32_t; };
 template <> struct CopyUnit<2> { using type = uint16_t; };
 
-constexpr int kRowsPerPass = 32;     // output rows whose sources a CTA resolves before copying them
-constexpr int kCopyUnroll = 8;       // copy units in flight per thread
+#ifndef TTF_COPY_UNROLL
+#define TTF_COPY_UNROLL 8
+#endif
+constexpr int kCopyUnroll = TTF_COPY_UNROLL;   // 16-byte units in flight per lane (two steps for an 8 KB row)
+constexpr int kScanChunks = 4;       // frame counts per lane fetched at once by the warp-level frame search
 
 // Cell index of the n-th (0-based) retained token of one frame: a warp-wide rank/select over the keep flags.
 // All lanes must call with the same arguments; returns -1 if the frame holds fewer than n+1 retained tokens.
@@ -112,7 +115,10 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
     using U = typename CopyUnit<COPY_BYTES>::type;
     const int N = H * W;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    pdl_launch_dependents();                     // the next call's sweep may be scheduled; it waits for this grid
+    trace_mark(const_cast<int*>(hdr), 3, false);
     pdl_wait();                                  // keep flags, dst and survivor counts are complete
+    trace_mark(const_cast<int*>(hdr), 6, false);
     const int a = __ldcg(hdr + HDR_ANCHOR);
 
     // ---- bookkeeping CTAs: tokens fused into each anchor cell (gather-side, integer, fixed order) --------
@@ -137,89 +143,84 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
         return;
     }
 
-    // ---- exclusive prefix of preserved tokens per frame ------------------------------------------------
-    __shared__ int s_pre[kSmemPrefixMaxF + 1];
-    __shared__ int s_warp[kCopyWarps];
-    __shared__ int s_src[kRowsPerPass];
-    const int* pre;
-    if (F <= kSmemPrefixMaxF) {
-        // each thread scans a contiguous run of frames, runs are combined over the block in thread order
-        const int per = (F + kCopyWarps * 32 - 1) / (kCopyWarps * 32);
-        const int k0 = tid * per;
-        int sum = 0;
-        for (int k = k0; k < min(F, k0 + per); ++k) sum += (k != a) ? __ldcg(cnt + k) : 0;
-        int incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int n = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += n;
-        }
-        if (lane == 31) s_warp[w] = incl;
-        __syncthreads();
-        int woff = 0;
-        for (int ww = 0; ww < w; ++ww) woff += s_warp[ww];
-        int run = woff + incl - sum;
-        for (int k = k0; k < min(F, k0 + per); ++k) { s_pre[k] = run; run += (k != a) ? __ldcg(cnt + k) : 0; }
-        if (tid == kCopyWarps * 32 - 1) s_pre[F] = woff + incl;
-        __syncthreads();
-        pre = s_pre;
-    } else {
-        pre = gprefix;
-    }
-    const int P = pre[F];
-    const int L = N + P;                                   // L' = N + P (Eq. Lpre)
-    if (blockIdx.x == 0 && tid == 0) { *out_count = L; }
-
-    // ---- output-driven gather: this CTA owns a contiguous, balanced range of output rows ------------------
-    const int j_begin = (int)((long long)L * blockIdx.x / ncopy_blocks);
-    const int j_end = (int)((long long)L * (blockIdx.x + 1) / ncopy_blocks);
-    const int upr = (int)(row_bytes / COPY_BYTES);         // copy units per row
-    for (int jb = j_begin; jb < j_end; jb += kRowsPerPass) {
-        const int rows = min(kRowsPerPass, j_end - jb);
-        __syncthreads();                                   // previous pass has finished with s_src
-        // a) source token of every output row of the pass: one warp per row
-        for (int rr = w; rr < rows; rr += kCopyWarps) {
-            const int j = jb + rr;
-            int f;
-            if (j < N) f = a * N + j;                      // anchor rows first (Eq. xprime_stack)
-            else {
-                const int e = j - N;
-                int lo = 0, hi = F;                        // largest k with pre[k] <= e
-                while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (pre[mid] <= e) lo = mid; else hi = mid; }
-                const int i = select_in_frame(keep + (size_t)lo * N, N, e - pre[lo], lane);
-                f = i < 0 ? -1 : lo * N + i;               // -1 cannot happen when cnt matches keep
+    // ---- output-driven gather, one warp per output row, no block-level synchronisation -----------------------
+    // frame search: the frame that holds the e-th preserved source token (flat order, anchor frame skipped)
+    // and the number of preserved tokens before that frame.  Returns the total P when e is past the end.
+    auto find_frame = [&](int e, int& k_out, int& before) -> int {
+        int running = 0;
+        k_out = -1; before = 0;
+        if (F > kWarpPrefixMaxF) {                         // pre-scanned prefix: binary search
+            int lo = 0, hi = F;
+            const int P = __ldcg(gprefix + F);
+            if (e < P) {
+                while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (__ldcg(gprefix + mid) <= e) lo = mid; else hi = mid; }
+                k_out = lo; before = __ldcg(gprefix + lo);
             }
-            if (lane == 0) s_src[rr] = f;
-            if (lane < 3 && f >= 0) {                      // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
-                const int k = f / N, i = f - k * N, yy = i / W;
-                out_pos[(size_t)j * 3 + lane] = lane == 0 ? k : (lane == 1 ? yy : i - yy * W);
-            }
+            return P;
         }
-        __syncthreads();
-        // b) copy: consecutive threads move consecutive 16-byte units, several rows in flight per thread
-        const long long total = (long long)rows * upr;
-        for (long long base = tid; base < total; base += (long long)kCopyWarps * 32 * kCopyUnroll) {
-            U v[kCopyUnroll];
-            long long o[kCopyUnroll];
+        for (int base = 0; base < F; base += 32 * kScanChunks) {
+            int c[kScanChunks];
 #pragma unroll
-            for (int q = 0; q < kCopyUnroll; ++q) {
-                const long long u = base + (long long)q * kCopyWarps * 32;
-                o[q] = -1;
-                if (u < total) {
-                    const int rr = (int)(u / upr);
-                    const int off = (int)(u - (long long)rr * upr);
-                    const int f = s_src[rr];
-                    if (f >= 0) {
-                        v[q] = __ldcs(reinterpret_cast<const U*>(X + (size_t)f * row_bytes) + off);
-                        o[q] = (long long)(jb + rr) * upr + off;
-                    }
+            for (int q = 0; q < kScanChunks; ++q) {
+                const int k = base + q * 32 + lane;
+                c[q] = (k < F && k != a) ? __ldcg(cnt + k) : 0;
+            }
+#pragma unroll
+            for (int q = 0; q < kScanChunks; ++q) {
+                int incl = c[q];
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += v;
                 }
+                const int total = __shfl_sync(0xffffffffu, incl, 31);
+                if (k_out < 0 && e < running + total) {
+                    const unsigned m = __ballot_sync(0xffffffffu, running + incl > e);
+                    const int l = __ffs(m) - 1;
+                    k_out = base + q * 32 + l;
+                    before = running + __shfl_sync(0xffffffffu, incl - c[q], l);
+                }
+                running += total;
             }
+            if (k_out >= 0 && e >= 0) break;               // e < 0 asks for the total only
+        }
+        return running;
+    };
+
+    const int gw = blockIdx.x * kCopyWarps + w;            // global warp index
+    const int nw = ncopy_blocks * kCopyWarps;
+    if (gw == 0) {                                         // L' = N + P (Eq. Lpre)
+        int kk, bb;
+        const int P = find_frame(-1, kk, bb);
+        if (lane == 0) *out_count = N + P;
+    }
+    const int upr = (int)(row_bytes / COPY_BYTES);         // copy units per row
+    for (int j = gw; ; j += nw) {
+        int f;
+        if (j < N) f = a * N + j;                          // anchor rows first (Eq. xprime_stack)
+        else {
+            int k, before;
+            find_frame(j - N, k, before);
+            if (k < 0) break;                              // past the last output row
+            const int i = select_in_frame(keep + (size_t)k * N, N, j - N - before, lane);
+            if (i < 0) break;                              // cannot happen when cnt matches keep
+            f = k * N + i;
+        }
+        if (lane < 3) {                                    // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
+            const int k = f / N, i = f - k * N, yy = i / W;
+            out_pos[(size_t)j * 3 + lane] = lane == 0 ? k : (lane == 1 ? yy : i - yy * W);
+        }
+        const U* src = reinterpret_cast<const U*>(X + (size_t)f * row_bytes);
+        U* dsto = reinterpret_cast<U*>(out_tokens + (size_t)j * row_bytes);
+        for (int u0 = lane; u0 < upr; u0 += 32 * kCopyUnroll) {
+            U v[kCopyUnroll];
 #pragma unroll
-            for (int q = 0; q < kCopyUnroll; ++q)
-                if (o[q] >= 0) __stcs(reinterpret_cast<U*>(out_tokens) + o[q], v[q]);
+            for (int q = 0; q < kCopyUnroll; ++q) if (u0 + q * 32 < upr) v[q] = __ldcs(src + u0 + q * 32);
+#pragma unroll
+            for (int q = 0; q < kCopyUnroll; ++q) if (u0 + q * 32 < upr) __stcs(dsto + u0 + q * 32, v[q]);
         }
     }
+    trace_mark(const_cast<int*>(hdr), 3, true);
 }
 
 cudaError_t launch_fuse_count(const Problem& p, const Scratch& s, const int* dst, const unsigned char* keep,
@@ -237,12 +238,14 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
     const size_t esize = p.dtype == 0 ? 4 : 2;
     const size_t row_bytes = (size_t)p.C * esize;
     const bool vec = p.vec && (reinterpret_cast<uintptr_t>(out_tokens) % 16 == 0);
-    if (p.F > kSmemPrefixMaxF) {
+    if (p.F > kWarpPrefixMaxF) {
         k_frame_prefix<<<1, 1024, 0, st>>>(s.cnt, s.hdr, p.F, s.prefix);
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    const int ncopy = 2 * sm_count();
+    // enough warps for one output row each at the usual two-thirds removal (a warp loops when there are more)
+    const long long want = ((long long)p.F * p.N / 3 + p.N + kCopyWarps - 1) / kCopyWarps;
+    const int ncopy = (int)(want < 3LL * sm_count() ? (want < 1 ? 1 : want) : 3LL * sm_count());
     int nfuse = (p.N + kCopyWarps - 1) / kCopyWarps;
     if (nfuse > sm_count()) nfuse = sm_count();
     const int grid = ncopy + nfuse;
@@ -250,7 +253,7 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
     unsigned char* out = reinterpret_cast<unsigned char*>(out_tokens);
     const dim3 g(grid), b(kCopyWarps * 32);
     // the pre-scanned prefix of very long clips is read through plain loads: order that case by the stream
-    const bool pdl = p.F <= kSmemPrefixMaxF;
+    const bool pdl = p.F <= kWarpPrefixMaxF;
     if (vec)
         return launch_pdl_if(pdl, k_compact<16>, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
                           (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep, (const int*)s.dst,

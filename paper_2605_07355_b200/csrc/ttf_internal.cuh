@@ -9,7 +9,7 @@
 namespace ttf {
 
 constexpr float kNormFloor = 1e-12f;   // norms are floored here before dividing (zero token -> similarity 0)
-constexpr int kSmemPrefixMaxF = 2048;  // frame counts up to this are scanned in shared memory by the gather
+constexpr int kWarpPrefixMaxF = 1024;  // frame counts up to this are scanned by each warp of the gather itself
 constexpr int kHdrInts = 64;
 
 // header words of the scratch block
@@ -27,7 +27,7 @@ struct Problem {
     int cpt;            // norm sweep: chunks of lanes_elems channels per thread per row (1 or 2)
     int ncb;            // norm sweep: column blocks of 256 * cpt chunks per row
     int nslice;         // planes of partial squared norms: 8 warps x ncb
-    int nsl;            // anchor pick: channel slices (64 channels when C % 4 == 0, else 16)
+    int nsl;            // anchor pick: channel slices (32 channels when C % 4 == 0, else 8)
     int anchor_mode;    // 0 auto (Eq. auto_anchor), 1 first, 2 last, 3 explicit
     int anchor_arg;     // explicit anchor frame
 };
@@ -36,7 +36,7 @@ struct Problem {
 struct Scratch {
     int* hdr;           // [kHdrInts]  anchor frame, arrival counter of the anchor-pick slices
     int* cnt;           // [F]   preserved tokens per source frame (Eq. gating summed over a frame)
-    int* prefix;        // [F+1] exclusive scan of cnt, only used when F > kSmemPrefixMaxF
+    int* prefix;        // [F+1] exclusive scan of cnt, only used when F > kWarpPrefixMaxF
     float* fcos;        // [F]   cosine of each frame mean to the global mean (Eq. auto_anchor)
     float* Sp;          // [TG, F, C] per-frame channel sums of each token group
     float* Dp;          // [nsl, F] per-slice share of <S_k, g>
@@ -97,6 +97,21 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, c
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Development aid (compiled out unless TTF_TRACE is defined): earliest start / latest end of every kernel of
+// a call in nanoseconds of the global timer, kept in header words 16..47 of the scratch block.
+#ifdef TTF_TRACE
+__device__ __forceinline__ void trace_mark(int* hdr, int id, bool end) {
+    if (threadIdx.x == 0) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        unsigned long long* s = reinterpret_cast<unsigned long long*>(hdr + 16) + id * 2 + (end ? 1 : 0);
+        atomicMax(s, end ? t : ~t);
+    }
+}
+#else
+__device__ __forceinline__ void trace_mark(int*, int, bool) {}
+#endif
+
 struct bf16_t { uint16_t bits; };   // storage type only: all arithmetic is on the widened fp32 value
 
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
@@ -108,6 +123,7 @@ template <typename T, int V> struct Loader;
 template <> struct Loader<float, 4> {
     using Raw = float4;
     static __device__ __forceinline__ Raw load_raw(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+    static __device__ __forceinline__ Raw load_raw_cg(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
     static __device__ __forceinline__ Raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[4]) { x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
     static __device__ __forceinline__ void load(const float* p, float (&x)[4]) { unpack(load_raw(p), x); }
@@ -115,6 +131,7 @@ template <> struct Loader<float, 4> {
 template <> struct Loader<float, 1> {
     using Raw = float;
     static __device__ __forceinline__ Raw load_raw(const float* p) { return __ldg(p); }
+    static __device__ __forceinline__ Raw load_raw_cg(const float* p) { return __ldcg(p); }
     static __device__ __forceinline__ Raw zero() { return 0.f; }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[1]) { x[0] = v; }
     static __device__ __forceinline__ void load(const float* p, float (&x)[1]) { x[0] = __ldg(p); }
@@ -122,6 +139,7 @@ template <> struct Loader<float, 1> {
 template <> struct Loader<bf16_t, 8> {
     using Raw = uint4;
     static __device__ __forceinline__ Raw load_raw(const bf16_t* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+    static __device__ __forceinline__ Raw load_raw_cg(const bf16_t* p) { return __ldcg(reinterpret_cast<const uint4*>(p)); }
     static __device__ __forceinline__ Raw zero() { return make_uint4(0, 0, 0, 0); }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[8]) {
         x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);
@@ -133,6 +151,9 @@ template <> struct Loader<bf16_t, 1> {
     using Raw = float;
     static __device__ __forceinline__ Raw load_raw(const bf16_t* p) {
         return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short*>(p))) << 16);
+    }
+    static __device__ __forceinline__ Raw load_raw_cg(const bf16_t* p) {
+        return __uint_as_float(static_cast<uint32_t>(__ldcg(reinterpret_cast<const unsigned short*>(p))) << 16);
     }
     static __device__ __forceinline__ Raw zero() { return 0.f; }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[1]) { x[0] = v; }

@@ -158,7 +158,9 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int g = lane >> 2, tig = lane & 3;
     pdl_launch_dependents();
+    trace_mark(const_cast<int*>(hdr), 2, false);
     pdl_wait();                                  // norms and the anchor index are complete
+    trace_mark(const_cast<int*>(hdr), 5, false);
     const int a = __ldcg(hdr + HDR_ANCHOR);
     const int y = i / W, x = i - y * W;
     const int side = 2 * r + 1, ncand = side * side;
@@ -262,6 +264,7 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
             }
         }
     }
+    trace_mark(const_cast<int*>(hdr), 2, true);
 }
 
 template <int MT, int NT>
