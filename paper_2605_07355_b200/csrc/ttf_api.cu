@@ -64,8 +64,7 @@ void carve_scratch(const Problem& p, void* base, Scratch* s) {
     s->hdr = (int*)take(sizeof(int) * kHdrInts);      // control words first: one small memset clears them
     s->cnt = (int*)take(sizeof(int) * p.F);
     s->prefix = (int*)take(sizeof(int) * ((size_t)p.F + 1));
-    s->fcos = (float*)take(sizeof(float) * p.F);
-    s->Sp = (float*)take(sizeof(float) * (size_t)norm_token_groups(p) * p.F * p.C);
+    s->S = (float*)take(sizeof(float) * (size_t)p.F * p.C);
     s->Dp = (float*)take(sizeof(float) * (size_t)p.nsl * p.F);
     s->Qp = (float*)take(sizeof(float) * (size_t)p.nsl * p.F);
     s->Gp = (float*)take(sizeof(float) * (size_t)p.nsl);
@@ -92,11 +91,14 @@ static int make_problem(const void* X, int F, int H, int W, int C, int r, float 
     const long long row_bytes = (long long)C * esize;
     p->vec = (row_bytes % 16 == 0) && (reinterpret_cast<uintptr_t>(X) % 16 == 0);
     p->lanes_elems = p->vec ? (int)(16 / esize) : 1;
+    // norm sweep: 64-lane slices unless that leaves fewer than ~200 CTAs (shape-only rule: the order of every
+    // sum must not depend on the device)
     const long long chunks = ((long long)C + p->lanes_elems - 1) / p->lanes_elems;
-    p->cpt = chunks <= 256 ? 1 : 2;
-    p->ncb = (int)((chunks + 256LL * p->cpt - 1) / (256LL * p->cpt));
-    p->nslice = 8 * p->ncb;
-    p->nsl = C % 4 == 0 ? (C + 31) / 32 : (C + 7) / 8;
+    p->ls = ((chunks + 63) / 64) * F >= 192 ? 64 : 32;
+    p->nq = (int)((chunks + p->ls - 1) / p->ls);
+    p->nslice = p->nq * (p->ls / 32);
+    if ((long long)F * p->nq >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
+    p->nsl = C % 4 == 0 ? (C + 127) / 128 : (C + 31) / 32;
     p->anchor_mode = 0; p->anchor_arg = 0;
     return TTF_OK;
 }
@@ -150,7 +152,7 @@ static int run_front(const Problem& p, const Scratch& s, int* out_anchor, float*
     cudaError_t e;
     { ProfScope ps(st, PK_NORM_ANCHOR); e = launch_norm_anchor(p, s, out_anchor, st); }
     if (e != cudaSuccess) return cuda_fail(e);
-    { ProfScope ps(st, PK_MATCH); e = launch_match(p, s, shat, dst, keep, st); }
+    { ProfScope ps(st, PK_MATCH); e = launch_match(p, s, out_anchor, shat, dst, keep, st); }
     if (e != cudaSuccess) return cuda_fail(e);
     return TTF_OK;
 }

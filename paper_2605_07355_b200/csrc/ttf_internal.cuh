@@ -11,6 +11,7 @@ namespace ttf {
 constexpr float kNormFloor = 1e-12f;   // norms are floored here before dividing (zero token -> similarity 0)
 constexpr int kWarpPrefixMaxF = 1024;  // frame counts up to this are scanned by each warp of the gather itself
 constexpr int kHdrInts = 64;
+constexpr int kResolveMaxF = 256;      // clips up to this many frames: the matching kernel takes the arg max itself
 
 // header words of the scratch block
 enum { HDR_ANCHOR = 0, HDR_DONE_ALL = 1 };
@@ -24,10 +25,10 @@ struct Problem {
     int N;              // H * W
     int vec;            // 1 when rows are 16-byte aligned and a multiple of 16 bytes long, else 0
     int lanes_elems;    // channels one lane loads at once: 16 B worth when vec, else 1
-    int cpt;            // norm sweep: chunks of lanes_elems channels per thread per row (1 or 2)
-    int ncb;            // norm sweep: column blocks of 256 * cpt chunks per row
-    int nslice;         // planes of partial squared norms: 8 warps x ncb
-    int nsl;            // anchor pick: channel slices (32 channels when C % 4 == 0, else 8)
+    int ls;             // norm sweep: lanes across a channel slice (64, or 32 when that gives too few CTAs)
+    int nq;             // norm sweep: channel slices per row, ceil(C / (ls * lanes_elems))
+    int nslice;         // planes of partial squared norms: one per warp across a slice, nq * ls / 32
+    int nsl;            // frame statistics: channel slices (128 channels when C % 4 == 0, else 32)
     int anchor_mode;    // 0 auto (Eq. auto_anchor), 1 first, 2 last, 3 explicit
     int anchor_arg;     // explicit anchor frame
 };
@@ -37,8 +38,7 @@ struct Scratch {
     int* hdr;           // [kHdrInts]  anchor frame, arrival counter of the anchor-pick slices
     int* cnt;           // [F]   preserved tokens per source frame (Eq. gating summed over a frame)
     int* prefix;        // [F+1] exclusive scan of cnt, only used when F > kWarpPrefixMaxF
-    float* fcos;        // [F]   cosine of each frame mean to the global mean (Eq. auto_anchor)
-    float* Sp;          // [TG, F, C] per-frame channel sums of each token group
+    float* S;           // [F, C] per-frame channel sums
     float* Dp;          // [nsl, F] per-slice share of <S_k, g>
     float* Qp;          // [nsl, F] per-slice share of |S_k|^2
     float* Gp;          // [nsl]    per-slice share of |g|^2
@@ -50,20 +50,41 @@ struct Scratch {
     size_t bytes;       // total, multiple of 256
 };
 
+// Where a kernel gets the anchor frame a* from.
+struct AnchorSrc {
+    const float* Dp;    // [nsl, F] slice shares of <S_k, g>
+    const float* Qp;    // [nsl, F] slice shares of |S_k|^2
+    const float* Gp;    // [nsl]    slice shares of |g|^2
+    int nsl;
+    int fixed;          // >= 0: the anchor is this frame (first / last / explicit rule)
+    int from_hdr;       // 1: an earlier kernel left it in hdr[HDR_ANCHOR]
+    int* hdr;
+    int* out_anchor;    // optional user copy
+};
+
+inline AnchorSrc make_anchor_src(const Problem& p, const Scratch& s, int* out_anchor);
+
 // Fills the offsets (base may be NULL to only compute `bytes`).
 void carve_scratch(const Problem& p, void* base, Scratch* s);
 
 // Kernel launchers (each enqueues on `st` and returns the launch error, if any).
-int norm_token_groups(const Problem& p);   // token groups per frame of the norm/anchor sweep (shape-only rule)
 cudaError_t launch_norm_anchor(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st);
-cudaError_t launch_match(const Problem& p, const Scratch& s, float* shat, int* dst, unsigned char* keep,
-                         cudaStream_t st);
+cudaError_t launch_match(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
+                         unsigned char* keep, cudaStream_t st);
 cudaError_t launch_fuse_count(const Problem& p, const Scratch& s, const int* dst, const unsigned char* keep,
                               int* fuse_cnt, cudaStream_t st);
 cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens, int* out_pos, int* out_count,
                            cudaStream_t st);
 
 int sm_count();   // SMs of the current device (cached per device)
+
+inline AnchorSrc make_anchor_src(const Problem& p, const Scratch& s, int* out_anchor) {
+    AnchorSrc a;
+    a.Dp = s.Dp; a.Qp = s.Qp; a.Gp = s.Gp; a.nsl = p.nsl; a.hdr = s.hdr; a.out_anchor = out_anchor;
+    a.fixed = p.anchor_mode == 0 ? -1 : (p.anchor_mode == 1 ? 0 : (p.anchor_mode == 2 ? p.F - 1 : p.anchor_arg));
+    a.from_hdr = (p.anchor_mode == 0 && p.F > kResolveMaxF) ? 1 : 0;
+    return a;
+}
 
 // Launch with programmatic dependent launch: the kernel may be scheduled while the previous kernel of the
 // stream drains; it must execute pdl_wait() before it touches anything an earlier kernel wrote, and every
@@ -164,6 +185,57 @@ __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
+}
+
+// Anchor Frame Selection, last step (Eq. auto_anchor): a* = arg max_k <S_k, g> / (|S_k| |g|), lowest frame on
+// ties, from the per-slice shares written by k_frame_stats; the shares are added in slice order.  Called by
+// all threads of a CTA (any block size that is a multiple of 32, at most 1024); returns the same value to all.
+__device__ __forceinline__ int resolve_anchor(const AnchorSrc& src, int F) {
+    if (src.fixed >= 0) return src.fixed;
+    if (src.from_hdr) return __ldcg(src.hdr + HDR_ANCHOR);
+    __shared__ float s_d[32][33], s_q[32][33];        // [warp][frame of the chunk]
+    __shared__ int s_anchor;
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, nw = blockDim.x >> 5;
+    float ginv = 0.f;
+    if (w == 0) {
+        float gg = 0.f;
+        for (int q = lane; q < src.nsl; q += 32) gg += __ldcg(src.Gp + q);
+        gg = warp_sum(gg);
+        ginv = 1.0f / fmaxf(sqrtf(gg), kNormFloor);
+    }
+    float best = -INFINITY;
+    int idx = 0x7fffffff;
+    for (int kb = 0; kb < F; kb += 32) {              // lane = frame: loads are coalesced over the frames
+        const int kk = kb + lane;
+        float d = 0.f, s2 = 0.f;
+        if (kk < F) {
+#pragma unroll 4
+            for (int q = w; q < src.nsl; q += nw) {   // warp w adds the slices w, w + nw, ...
+                d += __ldcg(src.Dp + (size_t)q * F + kk);
+                s2 += __ldcg(src.Qp + (size_t)q * F + kk);
+            }
+        }
+        s_d[w][lane] = d; s_q[w][lane] = s2;
+        __syncthreads();
+        if (w == 0 && kk < F) {                       // warps combined in warp order
+            float dd = 0.f, qq = 0.f;
+            for (int ww = 0; ww < nw; ++ww) { dd += s_d[ww][lane]; qq += s_q[ww][lane]; }
+            const float v = dd * ginv * (1.0f / fmaxf(sqrtf(qq), kNormFloor));
+            if (v > best || idx == 0x7fffffff) { best = v; idx = kk; }   // ascending kk per lane: first max stays
+        }
+        __syncthreads();
+    }
+    if (w == 0) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+            if (oi != 0x7fffffff && (idx == 0x7fffffff || ob > best || (ob == best && oi < idx))) { best = ob; idx = oi; }
+        }
+        if (lane == 0) s_anchor = idx;
+    }
+    __syncthreads();
+    return s_anchor;
 }
 
 // 1 / max(||x||, floor) from the per-slice partial squared norms of token f, summed in slice order

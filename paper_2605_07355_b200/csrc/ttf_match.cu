@@ -19,17 +19,21 @@ constexpr int kMatchWarps = 8;
 template <typename T, int V>
 __global__ void __launch_bounds__(kMatchWarps * 32)
 k_match_generic(const T* __restrict__ X, int F, int H, int W, int C, int r, float t, int fchunk, int nslice,
-                const int* __restrict__ hdr, const float* __restrict__ ssq,
+                AnchorSrc asrc, const float* __restrict__ ssq,
                 float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep,
                 int* __restrict__ cnt)
 {
     pdl_launch_dependents();
-    pdl_wait();                                  // norms and the anchor index are complete
+    pdl_wait();                                  // norms and the frame statistics are complete
     const int N = H * W;
     const int i = blockIdx.x % N;
     const int chunk = blockIdx.x / N;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    const int a = __ldcg(hdr + HDR_ANCHOR);
+    const int a = resolve_anchor(asrc, F);
+    if (blockIdx.x == 0 && threadIdx.x == 0 && !asrc.from_hdr) {
+        asrc.hdr[HDR_ANCHOR] = a;                // the gather reads it from here
+        if (asrc.out_anchor) *asrc.out_anchor = a;
+    }
     const int y = i / W, x = i - y * W;
     const size_t FN = (size_t)F * N;
     const int y_lo = max(0, y - r), y_hi = min(H - 1, y + r);
@@ -140,7 +144,7 @@ __device__ __forceinline__ void mma_compute_stage(const MmaStage<MT, NT>& sg, fl
 template <int MT, int NT>
 __global__ void __launch_bounds__(kMmaWarps * 32, 2)
 k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t, int nslice,
-            const int* __restrict__ hdr, const float* __restrict__ ssq,
+            AnchorSrc asrc, const float* __restrict__ ssq,
             float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep,
             int* __restrict__ cnt)
 {
@@ -158,10 +162,22 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int g = lane >> 2, tig = lane & 3;
     pdl_launch_dependents();
-    trace_mark(const_cast<int*>(hdr), 2, false);
-    pdl_wait();                                  // norms and the anchor index are complete
-    trace_mark(const_cast<int*>(hdr), 5, false);
-    const int a = __ldcg(hdr + HDR_ANCHOR);
+    trace_mark(asrc.hdr, 2, false);
+#ifdef TTF_WARM
+    {   // rehearsal: run the anchor search once on whatever the buffers hold, only to have its code fetched
+        const int warm = resolve_anchor(asrc, F);
+        if (warm == 0x7ffffffe) asrc.hdr[kHdrInts - 1] = warm;
+        __syncthreads();
+    }
+#endif
+    pdl_wait();                                  // norms and the frame statistics are complete
+    trace_mark(asrc.hdr, 5, false);
+    const int a = resolve_anchor(asrc, F);
+    if (blockIdx.x == 0 && tid == 0 && !asrc.from_hdr) {
+        asrc.hdr[HDR_ANCHOR] = a;                // the gather reads it from here
+        if (asrc.out_anchor) *asrc.out_anchor = a;
+    }
+    trace_mark(asrc.hdr, 4, true);
     const int y = i / W, x = i - y * W;
     const int side = 2 * r + 1, ncand = side * side;
     const size_t FN = (size_t)F * N;
@@ -264,20 +280,20 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
             }
         }
     }
-    trace_mark(const_cast<int*>(hdr), 2, true);
+    trace_mark(asrc.hdr, 2, true);
 }
 
 template <int MT, int NT>
-static cudaError_t launch_mma_t(const Problem& p, const Scratch& s, float* shat, int* dst, unsigned char* keep,
-                                cudaStream_t st) {
+static cudaError_t launch_mma_t(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
+                                unsigned char* keep, cudaStream_t st) {
     const long long chunks = (p.F + 16 * MT - 1) / (16 * MT);
     return launch_pdl(k_match_mma<MT, NT>, dim3((unsigned)(chunks * p.N)), dim3(kMmaWarps * 32), st,
                       reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t, p.nslice,
-                      (const int*)s.hdr, (const float*)s.ssq, shat, dst, keep, s.cnt);
+                      make_anchor_src(p, s, out_anchor), (const float*)s.ssq, shat, dst, keep, s.cnt);
 }
 
 template <typename T, int V>
-static cudaError_t launch_generic_t(const Problem& p, const Scratch& s, float* shat, int* dst,
+static cudaError_t launch_generic_t(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                                     unsigned char* keep, cudaStream_t st) {
     // enough CTAs to fill the GPU a few times over: split the frames into chunks when the grid is small
     int fchunk = p.F;
@@ -290,20 +306,20 @@ static cudaError_t launch_generic_t(const Problem& p, const Scratch& s, float* s
     const long long nchunk = (p.F + fchunk - 1) / fchunk;
     return launch_pdl(k_match_generic<T, V>, dim3((unsigned)(nchunk * p.N)), dim3(kMatchWarps * 32), st,
                       reinterpret_cast<const T*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t, fchunk, p.nslice,
-                      (const int*)s.hdr, (const float*)s.ssq, shat, dst, keep, s.cnt);
+                      make_anchor_src(p, s, out_anchor), (const float*)s.ssq, shat, dst, keep, s.cnt);
 }
 
-cudaError_t launch_match(const Problem& p, const Scratch& s, float* shat, int* dst, unsigned char* keep,
-                         cudaStream_t st) {
-    if (p.dtype == 0) return p.vec ? launch_generic_t<float, 4>(p, s, shat, dst, keep, st)
-                                   : launch_generic_t<float, 1>(p, s, shat, dst, keep, st);
+cudaError_t launch_match(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
+                         unsigned char* keep, cudaStream_t st) {
+    if (p.dtype == 0) return p.vec ? launch_generic_t<float, 4>(p, s, out_anchor, shat, dst, keep, st)
+                                   : launch_generic_t<float, 1>(p, s, out_anchor, shat, dst, keep, st);
     if (p.vec && p.r <= 2 && (long long)p.N * ((p.F + 31) / 32) < (1LL << 31)) {
-        if (p.r == 0) return launch_mma_t<2, 1>(p, s, shat, dst, keep, st);
-        if (p.r == 1) return launch_mma_t<2, 2>(p, s, shat, dst, keep, st);
-        return launch_mma_t<2, 4>(p, s, shat, dst, keep, st);
+        if (p.r == 0) return launch_mma_t<2, 1>(p, s, out_anchor, shat, dst, keep, st);
+        if (p.r == 1) return launch_mma_t<2, 2>(p, s, out_anchor, shat, dst, keep, st);
+        return launch_mma_t<2, 4>(p, s, out_anchor, shat, dst, keep, st);
     }
-    return p.vec ? launch_generic_t<bf16_t, 8>(p, s, shat, dst, keep, st)
-                 : launch_generic_t<bf16_t, 1>(p, s, shat, dst, keep, st);
+    return p.vec ? launch_generic_t<bf16_t, 8>(p, s, out_anchor, shat, dst, keep, st)
+                 : launch_generic_t<bf16_t, 1>(p, s, out_anchor, shat, dst, keep, st);
 }
 
 }  // namespace ttf
