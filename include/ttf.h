@@ -79,7 +79,8 @@ int ttf_workspace_bytes(int F, int H, int W, int C, int r, int dtype, size_t* by
  *   out_tokens   [capacity F*H*W rows, C] same dtype as features; rows [0, N) are the anchor frame's tokens,
  *                rows [N, N+P) the preserved source tokens in ascending flat index k*N + i (Eq. xprime_stack).
  *   out_count    one int32: L' = N + P (Eq. Lpre).  pos_dec(l) = L' + T + l (Eq. decode_pos) is
- *                ttf_decode_pos below.
+ *                ttf_decode_pos below.  -1 reports that a kernel gave up on one of its (bounded) internal
+ *                waits, which does not happen on a healthy device; the other outputs are then undefined.
  *   out_pos_thw  [capacity F*H*W, 3] int32; row j = (k, y, x) of output row j (Eq. compress_pos).
  * Rows beyond L' are not written.  Scratch comes from a cache the library keeps per (device, stream),
  * allocated with cudaMalloc on first use and grown when a larger clip arrives; two calls on the same stream

@@ -1,10 +1,10 @@
 // Anchor Frame Selection (Eq. auto_anchor) and per-token norms: one streaming sweep over X plus a small
 // statistics kernel; the arg max itself is taken by the matching kernel's prologue (resolve_anchor).
 //
-// k_norm_sum.  A CTA owns (frame k, channel slice q); a slice is LS lanes x one 16-byte load (LS = 64: 1 KB
+// k_norm_sum.  A CTA owns (frame k, channel slice q); a slice is LS = 32 lanes x one 16-byte load (512 bytes
 // of every token row; the CTAs of neighbouring slices run side by side, so DRAM sees whole rows).  The
-// 256 / LS row groups of a CTA walk the tokens of the frame interleaved, eight tokens per thread in flight and
-// the next eight prefetched.  A thread keeps running sums of its channels; the row groups are combined through
+// 256 / LS row groups (warps) of a CTA walk the tokens of the frame interleaved, eight tokens per thread in
+// flight and the next eight prefetched.  A thread keeps running sums of its channels; the row groups are combined through
 // shared memory in a fixed order and give the frame sum S_k[slice] (= N x mean token of frame k) directly.
 // The squared norm of every token restricted to one warp's 32 lanes is reduced with a 9-shuffle fold and
 // stored as a partial (consumers add the partials in plane order).
@@ -18,7 +18,10 @@ namespace ttf {
 
 constexpr int kNormWarps = 8;
 constexpr int kNormThreads = kNormWarps * 32;
-constexpr int kBatch = 8;            // tokens per thread in flight (times two with the prefetch)
+#ifndef TTF_BATCH
+#define TTF_BATCH 8
+#endif
+constexpr int kBatch = TTF_BATCH;    // tokens per thread in flight (times two with the prefetch): 8 or 16
 
 // Sum of v[u] over the warp for u = 0..7 with 9 shuffles.  On return the lanes with (lane & 3) == 0 hold the
 // total of token u = 4*bit4 + 2*bit3 + bit2 of their lane index.
@@ -53,8 +56,9 @@ __device__ __forceinline__ float fold8(float (&v)[8], int lane) {
     return r;
 }
 
-// LS: lanes across a slice (32 or 64); RG = 256 / LS row groups walk the tokens interleaved
-template <typename T, int V, int LS>
+// LS: lanes across a slice (32 or 64); RG = 256 / LS row groups walk the tokens interleaved.
+// NORMS: also store the per-token partial squared norms (only the CUDA-core matching kernel reads them).
+template <typename T, int V, int LS, bool NORMS>
 __global__ void __launch_bounds__(kNormThreads)
 k_norm_sum(const T* __restrict__ X, int F, int N, int C, int nq,
            float* __restrict__ S, float* __restrict__ ssq, int* __restrict__ cnt, int* __restrict__ hdr)
@@ -101,12 +105,23 @@ k_norm_sum(const T* __restrict__ X, int F, int N, int C, int nq,
             L::unpack(cur[u], x);
             float s = 0.f;
 #pragma unroll
-            for (int v = 0; v < V; ++v) { s = fmaf(x[v], x[v], s); col[v] += x[v]; }
+            for (int v = 0; v < V; ++v) {
+                if (NORMS) s = fmaf(x[v], x[v], s);
+                col[v] += x[v];
+            }
             ss[u] = s;
         }
-        const float tot = fold8(ss, lane);
-        const int u = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
-        if ((lane & 3) == 0 && i0 + u * RG < N) plane[i0 + u * RG] = tot;
+        if (NORMS) {
+#pragma unroll
+            for (int h = 0; h < kBatch / 8; ++h) {
+                float part[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) part[e] = ss[h * 8 + e];
+                const float tot = fold8(part, lane);
+                const int u = h * 8 + ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+                if ((lane & 3) == 0 && i0 + u * RG < N) plane[i0 + u * RG] = tot;
+            }
+        }
 #pragma unroll
         for (int uu = 0; uu < kBatch; ++uu) cur[uu] = nxt[uu];
     }
@@ -131,11 +146,10 @@ template <typename T, int V>
 static cudaError_t launch_sum_t(const Problem& p, const Scratch& s, cudaStream_t st) {
     const T* X = reinterpret_cast<const T*>(p.X);
     const unsigned blocks = (unsigned)((long long)p.F * p.nq);
-    if (p.ls == 64)
-        return launch_pdl(k_norm_sum<T, V, 64>, dim3(blocks), dim3(kNormThreads), st, X, p.F, p.N, p.C, p.nq,
-                          s.S, s.ssq, s.cnt, s.hdr);
-    return launch_pdl(k_norm_sum<T, V, 32>, dim3(blocks), dim3(kNormThreads), st, X, p.F, p.N, p.C, p.nq,
-                      s.S, s.ssq, s.cnt, s.hdr);
+    const dim3 g(blocks), b(kNormThreads);
+    if (uses_mma_match(p))
+        return launch_pdl(k_norm_sum<T, V, 32, false>, g, b, st, X, p.F, p.N, p.C, p.nq, s.S, s.ssq, s.cnt, s.hdr);
+    return launch_pdl(k_norm_sum<T, V, 32, true>, g, b, st, X, p.F, p.N, p.C, p.nq, s.S, s.ssq, s.cnt, s.hdr);
 }
 
 // ---------------------------------------------------------------------------------------------------------

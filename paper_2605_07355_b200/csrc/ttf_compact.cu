@@ -9,6 +9,7 @@
 // with all of its 16-byte loads in flight at once, so the work per warp is the same no matter how unevenly
 // the survivors are spread over the frames.  No warp ever waits for another one.
 #include "ttf_internal.cuh"
+#include "ttf_async.cuh"
 
 namespace ttf {
 
@@ -67,6 +68,76 @@ template <> struct CopyUnit<2> { using type = uint16_t; };
 constexpr int kCopyUnroll = TTF_COPY_UNROLL;   // 16-byte units in flight per lane (two steps for an 8 KB row)
 constexpr int kScanChunks = 4;       // frame counts per lane fetched at once by the warp-level frame search
 
+// Tokens fused into each anchor cell j: |{(k,i): k != a, keep = 0, dst = j}|, gather-side (every cell looks at
+// the (2r+1)^2 x (F-1) tokens that can point to it), integer, fixed order.  Run by whole CTAs: block `b` of `nb`.
+__device__ __forceinline__ void fuse_count_cta(int F, int H, int W, int r, int a, const unsigned char* keep,
+                                               const int* dst, int* fuse_cnt, int b, int nb) {
+    if (fuse_cnt == nullptr) return;
+    const int N = H * W;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    for (int j = b * kCopyWarps + w; j < N; j += nb * kCopyWarps) {
+        const int y = j / W, x = j - y * W;
+        int c = 0;
+        for (int k = lane; k < F; k += 32) {
+            if (k == a) continue;
+            for (int yy = max(0, y - r); yy <= min(H - 1, y + r); ++yy)
+                for (int xx = max(0, x - r); xx <= min(W - 1, x + r); ++xx) {
+                    const size_t f = (size_t)k * N + yy * W + xx;
+                    c += (!__ldcg(keep + f) && __ldcg(dst + f) == j) ? 1 : 0;
+                }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+        if (lane == 0) fuse_cnt[j] = c;
+    }
+}
+
+// Frame search of the gather: the frame that holds the e-th preserved source token (flat order, anchor frame
+// skipped) and the number of preserved tokens before that frame.  Returns the total P; k_out = -1 when e is past
+// the end (e < 0 asks for the total only).  All lanes of a warp call it with the same arguments.
+__device__ __forceinline__ int find_frame(const int* __restrict__ cnt, const int* __restrict__ gprefix, int F, int a,
+                                          int lane, int e, int& k_out, int& before) {
+    int running = 0;
+    k_out = -1; before = 0;
+    if (F > kWarpPrefixMaxF) {                         // pre-scanned prefix: binary search
+        int lo = 0, hi = F;
+        const int P = __ldcg(gprefix + F);
+        if (e < P) {
+            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (__ldcg(gprefix + mid) <= e) lo = mid; else hi = mid; }
+            k_out = lo; before = __ldcg(gprefix + lo);
+        }
+        return P;
+    }
+    for (int base = 0; base < F; base += 32 * kScanChunks) {
+        int c[kScanChunks];
+#pragma unroll
+        for (int q = 0; q < kScanChunks; ++q) {
+            const int k = base + q * 32 + lane;
+            c[q] = (k < F && k != a) ? __ldcg(cnt + k) : 0;
+        }
+#pragma unroll
+        for (int q = 0; q < kScanChunks; ++q) {
+            int incl = c[q];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int v = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += v;
+            }
+            const int total = __shfl_sync(0xffffffffu, incl, 31);
+            if (k_out < 0 && e < running + total) {
+                const unsigned m = __ballot_sync(0xffffffffu, running + incl > e);
+                const int l = __ffs(m) - 1;
+                k_out = base + q * 32 + l;
+                before = running + __shfl_sync(0xffffffffu, incl - c[q], l);
+            }
+            running += total;
+        }
+        if (k_out >= 0 && e >= 0) break;               // e < 0 asks for the total only
+    }
+    return running;
+}
+
+
 // Cell index of the n-th (0-based) retained token of one frame: a warp-wide rank/select over the keep flags.
 // All lanes must call with the same arguments; returns -1 if the frame holds fewer than n+1 retained tokens.
 __device__ __forceinline__ int select_in_frame(const unsigned char* __restrict__ kf, int N, int n, int lane) {
@@ -104,6 +175,81 @@ __device__ __forceinline__ int select_in_frame(const unsigned char* __restrict__
     return -1;
 }
 
+// Gather with bulk asynchronous copies, for rows that are 16-byte aligned multiples of 16 bytes: a warp finds the
+// source row of its output row as above, then one lane moves the row global -> shared -> global with two bulk
+// copies per piece of at most kBulkPiece bytes, so no data passes through registers.
+constexpr int kBulkPiece = 8192;
+
+__global__ void __launch_bounds__(kCopyWarps * 32)
+k_compact_bulk(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, int W, int r,
+               const int* __restrict__ hdr, const int* __restrict__ cnt, const int* __restrict__ gprefix,
+               const unsigned char* __restrict__ keep, const int* __restrict__ dst,
+               unsigned char* __restrict__ out_tokens, int* __restrict__ out_pos, int* __restrict__ out_count,
+               int* __restrict__ fuse_cnt, int ncopy_blocks)
+{
+    extern __shared__ __align__(128) unsigned char stage[];     // [kCopyWarps][kBulkPiece]
+    __shared__ uint64_t bar[kCopyWarps];
+    const int N = H * W;
+    const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
+    pdl_launch_dependents();                     // the next call's sweep may be scheduled; it waits for this grid
+    trace_mark(const_cast<int*>(hdr), 3, false);
+    if (lane == 0) { mbar_init(&bar[w], 1); mbar_init_fence(); }
+    __syncwarp();
+    pdl_wait();                                  // keep flags and survivor counts are complete
+    trace_mark(const_cast<int*>(hdr), 6, false);
+    const int a = __ldcg(hdr + HDR_ANCHOR);
+    if ((int)blockIdx.x >= ncopy_blocks) {       // bookkeeping CTAs: tokens fused into each anchor cell
+        fuse_count_cta(F, H, W, r, a, keep, dst, fuse_cnt, (int)blockIdx.x - ncopy_blocks, (int)gridDim.x - ncopy_blocks);
+        return;
+    }
+    const int gw = blockIdx.x * kCopyWarps + w;
+    const int nw = ncopy_blocks * kCopyWarps;
+    if (gw == 0) {                               // L' = N + P (Eq. Lpre)
+        int kk, bb;
+        const int P = find_frame(cnt, gprefix, F, a, lane, -1, kk, bb);
+        if (lane == 0) *out_count = __ldcg(hdr + HDR_ERROR) ? -1 : N + P;
+    }
+    unsigned char* buf = stage + (size_t)w * kBulkPiece;
+    const int pieces = (int)((row_bytes + kBulkPiece - 1) / kBulkPiece);
+    uint32_t phase = 0;
+    bool gave_up = false;
+    for (int j = gw; ; j += nw) {
+        int f;
+        if (j < N) f = a * N + j;                // anchor rows first (Eq. xprime_stack)
+        else {
+            int k, before;
+            find_frame(cnt, gprefix, F, a, lane, j - N, k, before);
+            if (k < 0) break;                    // past the last output row
+            const int i = select_in_frame(keep + (size_t)k * N, N, j - N - before, lane);
+            if (i < 0) break;                    // cannot happen when cnt matches keep
+            f = k * N + i;
+        }
+        if (lane < 3) {                          // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
+            const int k = f / N, i = f - k * N, yy = i / W;
+            out_pos[(size_t)j * 3 + lane] = lane == 0 ? k : (lane == 1 ? yy : i - yy * W);
+        }
+        if (lane == 0 && !gave_up) {
+            for (int pc = 0; pc < pieces; ++pc) {
+                const size_t off = (size_t)pc * kBulkPiece;
+                const uint32_t bytes = (uint32_t)(row_bytes - off < (size_t)kBulkPiece ? row_bytes - off : kBulkPiece);
+                bulk_wait_read<0>();             // the previous store has finished reading the buffer
+                mbar_arrive_expect_tx(&bar[w], bytes);
+                bulk_load(buf, X + (size_t)f * row_bytes + off, bytes, &bar[w]);
+                if (!mbar_wait(&bar[w], phase & 1)) { gave_up = true; break; }
+                ++phase;
+                bulk_store(out_tokens + (size_t)j * row_bytes + off, buf, bytes);
+                bulk_commit();
+            }
+        }
+        __syncwarp();
+    }
+    if (lane == 0) {
+        bulk_wait<0>();                          // all rows of this warp are in global memory
+        if (gave_up) atomicExch(const_cast<int*>(hdr) + HDR_ERROR, 1);
+    }
+    trace_mark(const_cast<int*>(hdr), 3, true);
+}
+
 template <int COPY_BYTES>
 __global__ void __launch_bounds__(kCopyWarps * 32)
 k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, int W, int r,
@@ -121,78 +267,22 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
     trace_mark(const_cast<int*>(hdr), 6, false);
     const int a = __ldcg(hdr + HDR_ANCHOR);
 
-    // ---- bookkeeping CTAs: tokens fused into each anchor cell (gather-side, integer, fixed order) --------
+    // ---- bookkeeping CTAs: tokens fused into each anchor cell ------------------------------------------------
     if ((int)blockIdx.x >= ncopy_blocks) {
-        if (fuse_cnt == nullptr) return;
-        const int nb = gridDim.x - ncopy_blocks;
-        for (int j = ((int)blockIdx.x - ncopy_blocks) * kCopyWarps + w; j < N; j += nb * kCopyWarps) {
-            const int y = j / W, x = j - y * W;
-            int c = 0;
-            for (int k = lane; k < F; k += 32) {
-                if (k == a) continue;
-                for (int yy = max(0, y - r); yy <= min(H - 1, y + r); ++yy)
-                    for (int xx = max(0, x - r); xx <= min(W - 1, x + r); ++xx) {
-                        const size_t f = (size_t)k * N + yy * W + xx;
-                        c += (!__ldcg(keep + f) && __ldcg(dst + f) == j) ? 1 : 0;
-                    }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-            if (lane == 0) fuse_cnt[j] = c;
-        }
+        fuse_count_cta(F, H, W, r, a, keep, dst, fuse_cnt, (int)blockIdx.x - ncopy_blocks, (int)gridDim.x - ncopy_blocks);
         return;
     }
 
     // ---- output-driven gather, one warp per output row, no block-level synchronisation -----------------------
     // frame search: the frame that holds the e-th preserved source token (flat order, anchor frame skipped)
     // and the number of preserved tokens before that frame.  Returns the total P when e is past the end.
-    auto find_frame = [&](int e, int& k_out, int& before) -> int {
-        int running = 0;
-        k_out = -1; before = 0;
-        if (F > kWarpPrefixMaxF) {                         // pre-scanned prefix: binary search
-            int lo = 0, hi = F;
-            const int P = __ldcg(gprefix + F);
-            if (e < P) {
-                while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (__ldcg(gprefix + mid) <= e) lo = mid; else hi = mid; }
-                k_out = lo; before = __ldcg(gprefix + lo);
-            }
-            return P;
-        }
-        for (int base = 0; base < F; base += 32 * kScanChunks) {
-            int c[kScanChunks];
-#pragma unroll
-            for (int q = 0; q < kScanChunks; ++q) {
-                const int k = base + q * 32 + lane;
-                c[q] = (k < F && k != a) ? __ldcg(cnt + k) : 0;
-            }
-#pragma unroll
-            for (int q = 0; q < kScanChunks; ++q) {
-                int incl = c[q];
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += v;
-                }
-                const int total = __shfl_sync(0xffffffffu, incl, 31);
-                if (k_out < 0 && e < running + total) {
-                    const unsigned m = __ballot_sync(0xffffffffu, running + incl > e);
-                    const int l = __ffs(m) - 1;
-                    k_out = base + q * 32 + l;
-                    before = running + __shfl_sync(0xffffffffu, incl - c[q], l);
-                }
-                running += total;
-            }
-            if (k_out >= 0 && e >= 0) break;               // e < 0 asks for the total only
-        }
-        return running;
-    };
-
     const int gw = blockIdx.x * kCopyWarps + w;            // global warp index
     const int nw = ncopy_blocks * kCopyWarps;
     if (gw == 0) {                                         // L' = N + P (Eq. Lpre)
         int kk, bb;
-        const int P = find_frame(-1, kk, bb);
-        if (lane == 0) *out_count = N + P;
+        const int P = find_frame(cnt, gprefix, F, a, lane, -1, kk, bb);
+        // a bounded wait of an earlier kernel of this call gave up: report instead of a plausible count
+        if (lane == 0) *out_count = __ldcg(hdr + HDR_ERROR) ? -1 : N + P;
     }
     const int upr = (int)(row_bytes / COPY_BYTES);         // copy units per row
     for (int j = gw; ; j += nw) {
@@ -200,7 +290,7 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
         if (j < N) f = a * N + j;                          // anchor rows first (Eq. xprime_stack)
         else {
             int k, before;
-            find_frame(j - N, k, before);
+            find_frame(cnt, gprefix, F, a, lane, j - N, k, before);
             if (k < 0) break;                              // past the last output row
             const int i = select_in_frame(keep + (size_t)k * N, N, j - N - before, lane);
             if (i < 0) break;                              // cannot happen when cnt matches keep
@@ -254,10 +344,24 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
     const dim3 g(grid), b(kCopyWarps * 32);
     // the pre-scanned prefix of very long clips is read through plain loads: order that case by the stream
     const bool pdl = p.F <= kWarpPrefixMaxF;
-    if (vec)
-        return launch_pdl_if(pdl, k_compact<16>, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
-                          (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep, (const int*)s.dst,
-                          out, out_pos, out_count, s.fuse_cnt, ncopy);
+    if (vec) {
+        static bool configured = false;          // the attribute belongs to the function, set it once
+        const size_t smem = (size_t)kCopyWarps * kBulkPiece;
+        if (!configured) {
+            cudaError_t e = cudaFuncSetAttribute(k_compact_bulk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            configured = true;
+        }
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = g; cfg.blockDim = b; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
+        return cudaLaunchKernelEx(&cfg, k_compact_bulk, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
+                                  (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep,
+                                  (const int*)s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy);
+    }
     if (esize == 4)
         return launch_pdl_if(pdl, k_compact<4>, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
                           (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep, (const int*)s.dst,

@@ -14,7 +14,7 @@ constexpr int kHdrInts = 64;
 constexpr int kResolveMaxF = 256;      // clips up to this many frames: the matching kernel takes the arg max itself
 
 // header words of the scratch block
-enum { HDR_ANCHOR = 0, HDR_DONE_ALL = 1 };
+enum { HDR_ANCHOR = 0, HDR_DONE_ALL = 1, HDR_ERROR = 2 };   // HDR_ERROR: a bounded wait gave up
 
 // Problem description handed to every launcher.
 struct Problem {
@@ -63,6 +63,12 @@ struct AnchorSrc {
 };
 
 inline AnchorSrc make_anchor_src(const Problem& p, const Scratch& s, int* out_anchor);
+
+// bf16 clips with 16-byte aligned rows and r <= 2 take the tensor-core matching kernel, which also derives the
+// token norms itself; everything else takes the CUDA-core kernel, which reads the norms of the sweep.
+inline bool uses_mma_match(const Problem& p) {
+    return p.dtype == 1 && p.vec && p.r <= 2 && (long long)p.N * ((p.F + 15) / 16) < (1LL << 31);
+}
 
 // Fills the offsets (base may be NULL to only compute `bytes`).
 void carve_scratch(const Problem& p, void* base, Scratch* s);

@@ -130,21 +130,39 @@ __device__ __forceinline__ void mma_load_stage(MmaStage<MT, NT>& sg, const uint4
     for (int nt = 0; nt < NT; ++nt) sg.b[nt] = (ok && bvalid[nt]) ? __ldg(brow[nt] + idx) : make_uint4(0, 0, 0, 0);
 }
 
+// Dot products of the stage, plus the squared norms of all its rows: the Gram tile of a 16-row tile with
+// itself has the squared norms on its diagonal, so two extra MMAs per tile (columns = rows 0..7, then rows
+// 8..15) give them on the tensor pipe from the fragments that are in registers anyway.
 template <int MT, int NT>
-__device__ __forceinline__ void mma_compute_stage(const MmaStage<MT, NT>& sg, float (&acc)[MT][NT][4]) {
+__device__ __forceinline__ void mma_compute_stage(const MmaStage<MT, NT>& sg, float (&acc)[MT][NT][4],
+                                                  float (&accn)[MT][2][4], float (&accb)[NT][4]) {
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
             mma_bf16_16816(acc[mt][nt], sg.a[mt][0].x, sg.a[mt][1].x, sg.a[mt][0].y, sg.a[mt][1].y, sg.b[nt].x, sg.b[nt].y);
             mma_bf16_16816(acc[mt][nt], sg.a[mt][0].z, sg.a[mt][1].z, sg.a[mt][0].w, sg.a[mt][1].w, sg.b[nt].z, sg.b[nt].w);
         }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            mma_bf16_16816(accn[mt][h], sg.a[mt][0].x, sg.a[mt][1].x, sg.a[mt][0].y, sg.a[mt][1].y, sg.a[mt][h].x, sg.a[mt][h].y);
+            mma_bf16_16816(accn[mt][h], sg.a[mt][0].z, sg.a[mt][1].z, sg.a[mt][0].w, sg.a[mt][1].w, sg.a[mt][h].z, sg.a[mt][h].w);
+        }
+    }
+    // candidate rows: rows of the Gram tile = slots of the tile pair (even, odd), columns = slots of tile nt
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        const uint4 lo = sg.b[nt & ~1];
+        const uint4 hi = (nt | 1) < NT ? sg.b[(nt | 1) < NT ? (nt | 1) : nt] : make_uint4(0, 0, 0, 0);
+        mma_bf16_16816(accb[nt], lo.x, hi.x, lo.y, hi.y, sg.b[nt].x, sg.b[nt].y);
+        mma_bf16_16816(accb[nt], lo.z, hi.z, lo.w, hi.w, sg.b[nt].z, sg.b[nt].w);
+    }
 }
 
 template <int MT, int NT>
 __global__ void __launch_bounds__(kMmaWarps * 32, 2)
-k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t, int nslice,
-            AnchorSrc asrc, const float* __restrict__ ssq,
+k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t,
+            AnchorSrc asrc,
             float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep,
             int* __restrict__ cnt)
 {
@@ -152,6 +170,8 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
     constexpr int NC = 8 * NT;       // candidate slots per CTA (>= (2r+1)^2)
     __shared__ float s_part[kMmaWarps][FR][NC];
     __shared__ float s_dot[FR][NC];
+    __shared__ float s_na[kMmaWarps][FR];        // partial squared norms of the source rows, per warp
+    __shared__ float s_nb[kMmaWarps][NC];        // ... of the candidate rows
     __shared__ float s_rs[FR];
     __shared__ float s_ra[NC];
     __shared__ int s_j[NC];
@@ -170,7 +190,7 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
         __syncthreads();
     }
 #endif
-    pdl_wait();                                  // norms and the frame statistics are complete
+    pdl_wait();                                  // the frame statistics are complete (X itself is an input)
     trace_mark(asrc.hdr, 5, false);
     const int a = resolve_anchor(asrc, F);
     if (blockIdx.x == 0 && tid == 0 && !asrc.from_hdr) {
@@ -180,7 +200,6 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
     trace_mark(asrc.hdr, 4, true);
     const int y = i / W, x = i - y * W;
     const int side = 2 * r + 1, ncand = side * side;
-    const size_t FN = (size_t)F * N;
     const int units = C / 8;                     // 16-byte units per row
 
     // candidate c = (dy + r) * side + (dx + r): ascending c is ascending anchor index among in-grid cells
@@ -190,14 +209,7 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
         return (yy >= 0 && yy < H && xx >= 0 && xx < W) ? yy * W + xx : -1;
     };
 
-    if (tid < NC) {
-        const int j = cand_index(tid);
-        s_j[tid] = j;
-        s_ra[tid] = j >= 0 ? inv_norm(ssq, nslice, FN, (size_t)a * N + j) : 0.f;
-    } else if (tid >= 64 && tid < 64 + FR) {
-        const int k = k0 + tid - 64;
-        s_rs[tid - 64] = k < F ? inv_norm(ssq, nslice, FN, (size_t)k * N + i) : 0.f;
-    }
+    if (tid < NC) s_j[tid] = cand_index(tid);
 
     const uint4* arow[MT][2];
 #pragma unroll
@@ -216,13 +228,18 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
         brow[nt] = reinterpret_cast<const uint4*>(X + ((size_t)a * N + (j >= 0 ? j : 0)) * C);
     }
 
-    float acc[MT][NT][4];
+    float acc[MT][NT][4], accn[MT][2][4], accb[NT][4];
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+    for (int q = 0; q < 4; ++q) {
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
+        for (int mt = 0; mt < MT; ++mt) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) acc[mt][nt][q] = 0.f;
+            for (int nt = 0; nt < NT; ++nt) acc[mt][nt][q] = 0.f;
+            accn[mt][0][q] = 0.f; accn[mt][1][q] = 0.f;
+        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) accb[nt][q] = 0.f;
+    }
 
     // split K: warp w takes 64-byte blocks w, w + 8, ...; two blocks are in flight per warp
     const int nblk = (units + 3) / 4;
@@ -232,10 +249,10 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
     for (; blk < nblk; blk += 2 * kMmaWarps) {
         const int nb1 = blk + kMmaWarps, nb2 = blk + 2 * kMmaWarps;
         if (nb1 < nblk) mma_load_stage<MT, NT>(s1, arow, brow, bvalid, nb1 * 4 + tig, units);
-        mma_compute_stage<MT, NT>(s0, acc);
+        mma_compute_stage<MT, NT>(s0, acc, accn, accb);
         if (nb1 < nblk) {
             if (nb2 < nblk) mma_load_stage<MT, NT>(s0, arow, brow, bvalid, nb2 * 4 + tig, units);
-            mma_compute_stage<MT, NT>(s1, acc);
+            mma_compute_stage<MT, NT>(s1, acc, accn, accb);
         }
     }
 
@@ -249,12 +266,31 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
             s_part[w][mt * 16 + g + 8][nt * 8 + 2 * tig] = acc[mt][nt][2];
             s_part[w][mt * 16 + g + 8][nt * 8 + 2 * tig + 1] = acc[mt][nt][3];
         }
+    // Gram diagonals: the lane with tig == g / 2 holds entry (g, g) in c0 / c1 and (g + 8, g) in c2 / c3
+    if (tig == (g >> 1)) {
+        const bool odd = g & 1;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            s_na[w][mt * 16 + g] = odd ? accn[mt][0][1] : accn[mt][0][0];          // frame g against column g
+            s_na[w][mt * 16 + 8 + g] = odd ? accn[mt][1][3] : accn[mt][1][2];      // frame g + 8 against column g
+        }
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)                  // slot nt*8 + g is row g of an even tile, row g + 8 of an odd one
+            s_nb[w][nt * 8 + g] = (nt & 1) ? (odd ? accb[nt][3] : accb[nt][2]) : (odd ? accb[nt][1] : accb[nt][0]);
+    }
     __syncthreads();
     for (int idx = tid; idx < FR * NC; idx += kMmaWarps * 32) {
         float d = 0.f;
 #pragma unroll
         for (int ww = 0; ww < kMmaWarps; ++ww) d += (&s_part[ww][0][0])[idx];
         (&s_dot[0][0])[idx] = d;
+    }
+    if (tid < FR + NC) {                                 // 1 / max(||x||, floor), warps added in warp order
+        float n2 = 0.f;
+#pragma unroll
+        for (int ww = 0; ww < kMmaWarps; ++ww) n2 += tid < FR ? s_na[ww][tid] : s_nb[ww][tid - FR];
+        const float rinv = 1.0f / fmaxf(sqrtf(n2), kNormFloor);
+        if (tid < FR) s_rs[tid] = rinv; else s_ra[tid - FR] = rinv;
     }
     __syncthreads();
 
@@ -288,8 +324,8 @@ static cudaError_t launch_mma_t(const Problem& p, const Scratch& s, int* out_anc
                                 unsigned char* keep, cudaStream_t st) {
     const long long chunks = (p.F + 16 * MT - 1) / (16 * MT);
     return launch_pdl(k_match_mma<MT, NT>, dim3((unsigned)(chunks * p.N)), dim3(kMmaWarps * 32), st,
-                      reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t, p.nslice,
-                      make_anchor_src(p, s, out_anchor), (const float*)s.ssq, shat, dst, keep, s.cnt);
+                      reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t,
+                      make_anchor_src(p, s, out_anchor), shat, dst, keep, s.cnt);
 }
 
 template <typename T, int V>
@@ -313,10 +349,10 @@ cudaError_t launch_match(const Problem& p, const Scratch& s, int* out_anchor, fl
                          unsigned char* keep, cudaStream_t st) {
     if (p.dtype == 0) return p.vec ? launch_generic_t<float, 4>(p, s, out_anchor, shat, dst, keep, st)
                                    : launch_generic_t<float, 1>(p, s, out_anchor, shat, dst, keep, st);
-    if (p.vec && p.r <= 2 && (long long)p.N * ((p.F + 31) / 32) < (1LL << 31)) {
+    if (uses_mma_match(p)) {
         if (p.r == 0) return launch_mma_t<2, 1>(p, s, out_anchor, shat, dst, keep, st);
         if (p.r == 1) return launch_mma_t<2, 2>(p, s, out_anchor, shat, dst, keep, st);
-        return launch_mma_t<2, 4>(p, s, out_anchor, shat, dst, keep, st);
+        return launch_mma_t<1, 4>(p, s, out_anchor, shat, dst, keep, st);     // 25 candidates: 16 frames per CTA
     }
     return p.vec ? launch_generic_t<bf16_t, 8>(p, s, out_anchor, shat, dst, keep, st)
                  : launch_generic_t<bf16_t, 1>(p, s, out_anchor, shat, dst, keep, st);
