@@ -168,7 +168,7 @@ constexpr int kStatSub = 1;
 
 template <int V>
 __global__ void __launch_bounds__(kNormThreads)
-k_frame_stats(const float* S, int F, int C, float* Dp, float* Qp, float* Gp, int* hdr)
+k_frame_stats(const float* S, int F, int C, int nsl, float* Dp, float* Qp, float* Gp, int* hdr)
 {
     pdl_launch_dependents();
     trace_mark(hdr, 1, false);
@@ -237,7 +237,10 @@ k_frame_stats(const float* S, int F, int C, float* Dp, float* Qp, float* Gp, int
             for (int v = 0; v < NV; ++v) { d = fmaf(acc[jj][v], gl[v], d); qq = fmaf(acc[jj][v], acc[jj][v], qq); }
             d = warp_sum(d);
             qq = warp_sum(qq);
-            if (lane == 0 && kk < F) { Dp[(size_t)q * F + kk] = d; Qp[(size_t)q * F + kk] = qq; }
+            if (lane < kStatReplicas && kk < F) {             // every lane holds the sums: one lane per replica
+                Dp[((size_t)lane * nsl + q) * F + kk] = d;
+                Qp[((size_t)lane * nsl + q) * F + kk] = qq;
+            }
         }
     }
     if (w == 0) {
@@ -245,7 +248,7 @@ k_frame_stats(const float* S, int F, int C, float* Dp, float* Qp, float* Gp, int
 #pragma unroll
         for (int v = 0; v < NV; ++v) gg = fmaf(gl[v], gl[v], gg);
         gg = warp_sum(gg);
-        if (lane == 0) Gp[q] = gg;
+        if (lane < kStatReplicas) Gp[(size_t)lane * nsl + q] = gg;
     }
     trace_mark(hdr, 1, true);
 }
@@ -267,10 +270,10 @@ cudaError_t launch_norm_anchor(const Problem& p, const Scratch& s, int* out_anch
     else e = p.vec ? launch_sum_t<bf16_t, 8>(p, s, st) : launch_sum_t<bf16_t, 1>(p, s, st);
     if (e != cudaSuccess || p.anchor_mode != 0) return e;      // fixed anchors need no statistics
     if (p.C % 4 == 0)
-        e = launch_pdl(k_frame_stats<4>, dim3(p.nsl), dim3(kNormThreads), st, (const float*)s.S, p.F, p.C,
+        e = launch_pdl(k_frame_stats<4>, dim3(p.nsl), dim3(kNormThreads), st, (const float*)s.S, p.F, p.C, p.nsl,
                        s.Dp, s.Qp, s.Gp, s.hdr);
     else
-        e = launch_pdl(k_frame_stats<1>, dim3(p.nsl), dim3(kNormThreads), st, (const float*)s.S, p.F, p.C,
+        e = launch_pdl(k_frame_stats<1>, dim3(p.nsl), dim3(kNormThreads), st, (const float*)s.S, p.F, p.C, p.nsl,
                        s.Dp, s.Qp, s.Gp, s.hdr);
     if (e != cudaSuccess) return e;
     if (p.F > kResolveMaxF) {

@@ -65,9 +65,9 @@ void carve_scratch(const Problem& p, void* base, Scratch* s) {
     s->cnt = (int*)take(sizeof(int) * p.F);
     s->prefix = (int*)take(sizeof(int) * ((size_t)p.F + 1));
     s->S = (float*)take(sizeof(float) * (size_t)p.F * p.C);
-    s->Dp = (float*)take(sizeof(float) * (size_t)p.nsl * p.F);
-    s->Qp = (float*)take(sizeof(float) * (size_t)p.nsl * p.F);
-    s->Gp = (float*)take(sizeof(float) * (size_t)p.nsl);
+    s->Dp = (float*)take(sizeof(float) * (size_t)kStatReplicas * p.nsl * p.F);
+    s->Qp = (float*)take(sizeof(float) * (size_t)kStatReplicas * p.nsl * p.F);
+    s->Gp = (float*)take(sizeof(float) * (size_t)kStatReplicas * p.nsl);
     s->ssq = (float*)take(sizeof(float) * (size_t)p.nslice * FN);
     s->shat = (float*)take(sizeof(float) * FN);
     s->dst = (int*)take(sizeof(int) * FN);

@@ -11,6 +11,8 @@ namespace ttf {
 constexpr float kNormFloor = 1e-12f;   // norms are floored here before dividing (zero token -> similarity 0)
 constexpr int kWarpPrefixMaxF = 1024;  // frame counts up to this are scanned by each warp of the gather itself
 constexpr int kHdrInts = 64;
+constexpr int kStatReplicas = 16;      // copies of the frame statistics, so that the CTAs that read them at the
+                                       // same moment do not all queue on the same few cache lines
 constexpr int kResolveMaxF = 256;      // clips up to this many frames: the matching kernel takes the arg max itself
 
 // header words of the scratch block
@@ -39,9 +41,9 @@ struct Scratch {
     int* cnt;           // [F]   preserved tokens per source frame (Eq. gating summed over a frame)
     int* prefix;        // [F+1] exclusive scan of cnt, only used when F > kWarpPrefixMaxF
     float* S;           // [F, C] per-frame channel sums
-    float* Dp;          // [nsl, F] per-slice share of <S_k, g>
-    float* Qp;          // [nsl, F] per-slice share of |S_k|^2
-    float* Gp;          // [nsl]    per-slice share of |g|^2
+    float* Dp;          // [kStatReplicas][nsl, F] per-slice share of <S_k, g>
+    float* Qp;          // [kStatReplicas][nsl, F] per-slice share of |S_k|^2
+    float* Gp;          // [kStatReplicas][nsl]    per-slice share of |g|^2
     float* ssq;         // [nslice, F*N] partial squared norms (one plane per warp and column block)
     float* shat;        // [F*N] best similarity (Eq. argmax)
     int* dst;           // [F*N] best anchor cell (Eq. dst)
@@ -52,9 +54,9 @@ struct Scratch {
 
 // Where a kernel gets the anchor frame a* from.
 struct AnchorSrc {
-    const float* Dp;    // [nsl, F] slice shares of <S_k, g>
-    const float* Qp;    // [nsl, F] slice shares of |S_k|^2
-    const float* Gp;    // [nsl]    slice shares of |g|^2
+    const float* Dp;    // [kStatReplicas][nsl, F] slice shares of <S_k, g>
+    const float* Qp;    // [kStatReplicas][nsl, F] slice shares of |S_k|^2
+    const float* Gp;    // [kStatReplicas][nsl]    slice shares of |g|^2
     int nsl;
     int fixed;          // >= 0: the anchor is this frame (first / last / explicit rule)
     int from_hdr;       // 1: an earlier kernel left it in hdr[HDR_ANCHOR]
@@ -202,10 +204,14 @@ __device__ __forceinline__ int resolve_anchor(const AnchorSrc& src, int F) {
     __shared__ float s_d[32][33], s_q[32][33];        // [warp][frame of the chunk]
     __shared__ int s_anchor;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5, nw = blockDim.x >> 5;
+    const int rep = blockIdx.x % kStatReplicas;       // identical copies: which one is read does not matter
+    const float* Dp = src.Dp + (size_t)rep * src.nsl * F;
+    const float* Qp = src.Qp + (size_t)rep * src.nsl * F;
+    const float* Gp = src.Gp + (size_t)rep * src.nsl;
     float ginv = 0.f;
     if (w == 0) {
         float gg = 0.f;
-        for (int q = lane; q < src.nsl; q += 32) gg += __ldcg(src.Gp + q);
+        for (int q = lane; q < src.nsl; q += 32) gg += __ldcg(Gp + q);
         gg = warp_sum(gg);
         ginv = 1.0f / fmaxf(sqrtf(gg), kNormFloor);
     }
@@ -217,8 +223,8 @@ __device__ __forceinline__ int resolve_anchor(const AnchorSrc& src, int F) {
         if (kk < F) {
 #pragma unroll 4
             for (int q = w; q < src.nsl; q += nw) {   // warp w adds the slices w, w + nw, ...
-                d += __ldcg(src.Dp + (size_t)q * F + kk);
-                s2 += __ldcg(src.Qp + (size_t)q * F + kk);
+                d += __ldcg(Dp + (size_t)q * F + kk);
+                s2 += __ldcg(Qp + (size_t)q * F + kk);
             }
         }
         s_d[w][lane] = d; s_q[w][lane] = s2;
