@@ -39,7 +39,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vl8b_cal")
     ap.add_argument("--clips", type=int, default=16, help="distinct clips per step (batch)")
-    ap.add_argument("--streams", type=int, default=1, help="CUDA streams the clips of a step are spread over")
+    ap.add_argument("--streams", type=int, default=4, help="CUDA streams the clips of a step are spread over")
     ap.add_argument("--threshold", type=float, default=None)
     ap.add_argument("--anchor", default="auto", choices=["auto", "first", "last"], help="anchor rule")
     ap.add_argument("--no-graph", action="store_true",

@@ -93,11 +93,14 @@ k_match_generic(const T* __restrict__ X, int F, int H, int W, int C, int r, floa
 // MMA (m16n8k16, fp32 accumulate: bf16 products are exact in fp32).  M = frames (16 per tile), N = candidates
 // (8 per tile), K = channels.
 //
-// No shared-memory staging: a dot product does not care about the order of its terms, so the K index of a
-// fragment may be any fixed permutation of the channels as long as A and B use the same one.  Each lane loads
+// No cross-thread staging: a dot product does not care about the order of its terms, so the K index of a
+// fragment may be any fixed permutation of the channels as long as A and B use the same one.  Each lane fetches
 // 16 contiguous bytes (8 channels) of "its" row (frame g / g+8 for A, candidate g for B; g = lane/4) at
 // 16-byte column lane%4 of a 64-byte block and uses them as its fragment elements of two consecutive MMA
-// steps.  Loads are therefore 128-bit, coalesced in 64-byte runs per row, and feed the MMA directly.
+// steps.  The fetch is a cp.async into a lane-private shared-memory slot (coalesced in 64-byte runs per row,
+// zero-filled past the row end and for absent candidates), several blocks ahead of the MMAs, so that the bytes
+// in flight are bounded by shared memory rather than by registers; the measured floor of this kernel is the
+// per-SM L2 read bandwidth (about 72 GB/s per SM), not latency.
 //
 // The 8 warps of a CTA take interleaved 64-byte blocks of the rows (split K) and their partial products are
 // summed through shared memory in warp order, so the result does not depend on scheduling.
@@ -110,24 +113,51 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
 }
 
 constexpr int kMmaWarps = 8;
+#ifndef TTF_MMA_STAGES
+#define TTF_MMA_STAGES 4
+#endif
+constexpr int kMmaStages = TTF_MMA_STAGES;       // cp.async stages per warp (kMmaStages - 1 blocks in flight)
 
+// One pipeline stage of a warp: the 16-byte fragment pieces of its 64-byte block, (2 MT + NT) per lane.  The
+// pieces travel global -> shared with cp.async (no registers are tied up while they are in flight, so a warp
+// keeps several stages outstanding); every lane copies into and later reads back its own 16-byte slots.
 template <int MT, int NT>
 struct MmaStage {
     uint4 a[MT][2];
     uint4 b[NT];
 };
 
+__device__ __forceinline__ void cp_async16(void* dst_smem, const void* src, bool valid) {
+    const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(dst_smem));
+    const int bytes = valid ? 16 : 0;            // 0 source bytes: the 16 destination bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// slot layout of a stage: [(2 MT + NT) pieces][32 lanes] x 16 bytes
 template <int MT, int NT>
-__device__ __forceinline__ void mma_load_stage(MmaStage<MT, NT>& sg, const uint4* const (&arow)[MT][2],
-                                               const uint4* const (&brow)[NT], const bool (&bvalid)[NT],
-                                               int idx, int units) {
+__device__ __forceinline__ void mma_issue_stage(uint4* slot, const uint4* const (&arow)[MT][2],
+                                                const uint4* const (&brow)[NT], const bool (&bvalid)[NT],
+                                                int idx, int units, int lane) {
     const bool ok = idx < units;
+    const int safe = ok ? idx : 0;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) sg.a[mt][h] = ok ? __ldg(arow[mt][h] + idx) : make_uint4(0, 0, 0, 0);
+        for (int h = 0; h < 2; ++h) cp_async16(slot + (mt * 2 + h) * 32 + lane, arow[mt][h] + safe, ok);
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) sg.b[nt] = (ok && bvalid[nt]) ? __ldg(brow[nt] + idx) : make_uint4(0, 0, 0, 0);
+    for (int nt = 0; nt < NT; ++nt) cp_async16(slot + (2 * MT + nt) * 32 + lane, brow[nt] + safe, ok && bvalid[nt]);
+}
+
+template <int MT, int NT>
+__device__ __forceinline__ void mma_read_stage(MmaStage<MT, NT>& sg, const uint4* slot, int lane) {
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) sg.a[mt][h] = slot[(mt * 2 + h) * 32 + lane];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) sg.b[nt] = slot[(2 * MT + nt) * 32 + lane];
 }
 
 // Dot products of the stage, plus the squared norms of all its rows: the Gram tile of a 16-row tile with
@@ -168,7 +198,13 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
 {
     constexpr int FR = 16 * MT;      // frames per CTA
     constexpr int NC = 8 * NT;       // candidate slots per CTA (>= (2r+1)^2)
-    __shared__ float s_part[kMmaWarps][FR][NC];
+    constexpr int PIECES = 2 * MT + NT;
+    // ring[warp][stage][piece][lane]; after the main loop the same memory holds the per-warp partial products
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    uint4* ring = reinterpret_cast<uint4*>(dyn_smem);
+    float (*s_part)[FR][NC] = reinterpret_cast<float (*)[FR][NC]>(dyn_smem);
+    static_assert(sizeof(float) * kMmaWarps * FR * NC <= sizeof(uint4) * kMmaWarps * kMmaStages * PIECES * 32,
+                  "partial products must fit the ring");
     __shared__ float s_dot[FR][NC];
     __shared__ float s_na[kMmaWarps][FR];        // partial squared norms of the source rows, per warp
     __shared__ float s_nb[kMmaWarps][NC];        // ... of the candidate rows
@@ -241,20 +277,29 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
         for (int nt = 0; nt < NT; ++nt) accb[nt][q] = 0.f;
     }
 
-    // split K: warp w takes 64-byte blocks w, w + 8, ...; two blocks are in flight per warp
+    // split K: warp w takes 64-byte blocks w, w + 8, ...; kMmaStages - 1 blocks are in flight per warp
     const int nblk = (units + 3) / 4;
-    MmaStage<MT, NT> s0, s1;
-    int blk = w;
-    if (blk < nblk) mma_load_stage<MT, NT>(s0, arow, brow, bvalid, blk * 4 + tig, units);
-    for (; blk < nblk; blk += 2 * kMmaWarps) {
-        const int nb1 = blk + kMmaWarps, nb2 = blk + 2 * kMmaWarps;
-        if (nb1 < nblk) mma_load_stage<MT, NT>(s1, arow, brow, bvalid, nb1 * 4 + tig, units);
-        mma_compute_stage<MT, NT>(s0, acc, accn, accb);
-        if (nb1 < nblk) {
-            if (nb2 < nblk) mma_load_stage<MT, NT>(s0, arow, brow, bvalid, nb2 * 4 + tig, units);
-            mma_compute_stage<MT, NT>(s1, acc, accn, accb);
-        }
+    uint4* wring = ring + (size_t)w * kMmaStages * PIECES * 32;
+    const int nmine = nblk > w ? (nblk - w + kMmaWarps - 1) / kMmaWarps : 0;      // blocks of this warp
+#pragma unroll
+    for (int st = 0; st < kMmaStages - 1; ++st) {
+        if (st < nmine)
+            mma_issue_stage<MT, NT>(wring + st * PIECES * 32, arow, brow, bvalid, (w + st * kMmaWarps) * 4 + tig, units, lane);
+        cp_async_commit();
     }
+    for (int b = 0; b < nmine; ++b) {
+        const int nb = b + kMmaStages - 1;
+        if (nb < nmine)
+            mma_issue_stage<MT, NT>(wring + (nb % kMmaStages) * PIECES * 32, arow, brow, bvalid,
+                                    (w + nb * kMmaWarps) * 4 + tig, units, lane);
+        cp_async_commit();
+        cp_async_wait<kMmaStages - 1>();         // block b has landed (each lane waits for its own copies)
+        MmaStage<MT, NT> sg;
+        mma_read_stage<MT, NT>(sg, wring + (b % kMmaStages) * PIECES * 32, lane);
+        mma_compute_stage<MT, NT>(sg, acc, accn, accb);
+    }
+    cp_async_wait<0>();
+    __syncthreads();                             // every warp is done with its ring: reuse it for the partials
 
     // accumulator fragment: c0,c1 = (frame g, candidates 2*tig, 2*tig+1); c2,c3 = (frame g+8, same candidates)
 #pragma unroll
@@ -323,9 +368,22 @@ template <int MT, int NT>
 static cudaError_t launch_mma_t(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                                 unsigned char* keep, cudaStream_t st) {
     const long long chunks = (p.F + 16 * MT - 1) / (16 * MT);
-    return launch_pdl(k_match_mma<MT, NT>, dim3((unsigned)(chunks * p.N)), dim3(kMmaWarps * 32), st,
-                      reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t,
-                      make_anchor_src(p, s, out_anchor), shat, dst, keep, s.cnt);
+    constexpr size_t smem = sizeof(uint4) * kMmaWarps * kMmaStages * (2 * MT + NT) * 32;
+    static bool configured = false;              // per instantiation; the attribute belongs to the function
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(k_match_mma<MT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(chunks * p.N)); cfg.blockDim = dim3(kMmaWarps * 32);
+    cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_match_mma<MT, NT>, reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C,
+                              p.r, p.t, make_anchor_src(p, s, out_anchor), shat, dst, keep, s.cnt);
 }
 
 template <typename T, int V>
