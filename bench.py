@@ -193,6 +193,20 @@ def reference_arm(args):
     print(json.dumps(line), flush=True)
 
 
+def combine_ranks(ms_local: float, tokens_local: int, device=None):
+    """Whole-job figures of a replica run: the slowest rank's time and the tokens of all ranks.  One clip never
+    spans ranks, so this all-reduce of two scalars after the timed region is the only communication there is."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms_local), int(tokens_local)
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    n = torch.tensor([tokens_local], dtype=torch.int64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(n, op=dist.ReduceOp.SUM)
+    return float(t.item()), int(n.item())
+
+
 def workload_config(spec, t, clips_per_step, streams, tokens_per_step, anchor="auto", graph=False):
     return {"workload": f"{spec.name}: F={spec.F} {spec.H}x{spec.W} C={spec.C} {spec.dtype} r={spec.r} t={t:.2f}",
             "generator": spec.family, "clips_per_step": clips_per_step, "tokens_per_step": tokens_per_step,
@@ -313,15 +327,11 @@ def main():
     e1.record(main_stream)
     barrier()
     w1 = time.perf_counter()
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        tmax = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms_total = float(tmax.item())
-    ms_step = ms_total / args.steps
     tokens_step = nclips * FN
-    value = world * tokens_step / (ms_step * 1e-3)
-    clips_per_s = world * nclips / (ms_step * 1e-3)
+    ms_total, tokens_all = combine_ranks(e0.elapsed_time(e1), tokens_step, dev)
+    ms_step = ms_total / args.steps
+    value = tokens_all / (ms_step * 1e-3)
+    clips_per_s = value / FN
 
     # ---- per-kernel durations: the same steps again with events around every launch -----------------------
     prof_steps = min(args.steps, 50)
@@ -368,11 +378,9 @@ def main():
                 d2h += L * (C * spec.itemsize + 12) + 4
         barrier()
         dt = time.perf_counter() - t0
-        if world > 1:
-            tm = torch.tensor([dt], dtype=torch.float64, device=dev)
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-            dt = float(tm.item())
-        e2e = {"value": world * tokens_step * args.e2e_steps / dt, "unit": UNIT,
+        dt_ms, tokens_e2e = combine_ranks(dt * 1e3, tokens_step * args.e2e_steps, dev)
+        dt = dt_ms * 1e-3
+        e2e = {"value": tokens_e2e / dt, "unit": UNIT,
                "h2d_bytes_per_step": nclips * clip_bytes, "d2h_bytes_per_step": d2h,
                "steps": args.e2e_steps, "api": "ttf_compress_host (pinned host buffers)"}
 
