@@ -170,11 +170,12 @@ int ttf_query_static(const void* features, int F, int H, int W, int C, int r, fl
  * ttf_profile_begin and ttf_profile_end every kernel this library launches is bracketed by two CUDA events
  * on its own stream.  ttf_profile_end waits for those events and returns, per kernel kind, the summed
  * device time in milliseconds and the number of launches; `kinds` is the length of both arrays
- * (TTF_KERNEL_KINDS covers all).  Kinds: 0 norm + frame-sum sweep with the anchor pick, 1 windowed match +
- * gate, 2 compaction gather (with the frame-count prefix of clips longer than 1024 frames), 3 fuse-count
- * bookkeeping of ttf_query.  Profiling is process-wide and meant for benchmarks; leave it off otherwise.
+ * (TTF_KERNEL_KINDS covers all).  Kinds: 0 frame-sum (and norm) sweep, 1 frame statistics of the anchor rule,
+ * 2 windowed match + gate (its prologue takes the anchor arg max), 3 compaction gather (with the frame-count
+ * prefix of clips longer than 1024 frames), 4 fuse-count bookkeeping of ttf_query.  Profiling is process-wide
+ * and meant for benchmarks; leave it off otherwise.
  */
-#define TTF_KERNEL_KINDS 4
+#define TTF_KERNEL_KINDS 5
 int ttf_profile_begin(void);
 int ttf_profile_end(double* total_ms, long long* launches, int kinds);
 

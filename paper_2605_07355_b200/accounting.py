@@ -31,8 +31,10 @@ def pass_bytes(F: int, N: int, C: int, itemsize: int, count: int) -> int:
 def kernel_bytes(kind: str, F: int, N: int, C: int, itemsize: int, count: int) -> int:
     """Algorithmic bytes of one launch of each kernel kind."""
     X = F * N * C * itemsize
-    if kind == "norm_anchor":       # reads X; writes the frame sums and one squared norm per token
-        return X + F * C * 4 + F * N * 4
+    if kind == "norm_sum":          # reads X; writes the frame sums (the norms only on the CUDA-core path)
+        return X + F * C * 4
+    if kind == "frame_stats":       # reads the frame sums
+        return F * C * 4
     if kind == "match":             # reads X (sources + anchor frame once); writes s_hat, dst, keep
         return X + F * N * 9
     if kind == "compact":           # reads the retained rows, writes them with their positions

@@ -25,7 +25,7 @@ EXPORTS = [
 ]
 TTF_ANCHOR_AUTO, TTF_ANCHOR_FIRST, TTF_ANCHOR_LAST, TTF_ANCHOR_EXPLICIT = 0, 1, 2, 3
 TTF_STATIC_SCRATCH_BYTES = 8 << 20
-KERNEL_KINDS = ["norm_anchor", "match", "compact", "fuse_count"]
+KERNEL_KINDS = ["norm_sum", "frame_stats", "match", "compact", "fuse_count"]
 
 _lib = None
 

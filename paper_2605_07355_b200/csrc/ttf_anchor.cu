@@ -264,11 +264,14 @@ k_anchor_final(AnchorSrc src, int F)
     }
 }
 
-cudaError_t launch_norm_anchor(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st) {
+cudaError_t launch_norm_sum(const Problem& p, const Scratch& s, cudaStream_t st) {
+    if (p.dtype == 0) return p.vec ? launch_sum_t<float, 4>(p, s, st) : launch_sum_t<float, 1>(p, s, st);
+    return p.vec ? launch_sum_t<bf16_t, 8>(p, s, st) : launch_sum_t<bf16_t, 1>(p, s, st);
+}
+
+cudaError_t launch_frame_stats(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st) {
+    if (p.anchor_mode != 0) return cudaSuccess;                // fixed anchors need no statistics
     cudaError_t e;
-    if (p.dtype == 0) e = p.vec ? launch_sum_t<float, 4>(p, s, st) : launch_sum_t<float, 1>(p, s, st);
-    else e = p.vec ? launch_sum_t<bf16_t, 8>(p, s, st) : launch_sum_t<bf16_t, 1>(p, s, st);
-    if (e != cudaSuccess || p.anchor_mode != 0) return e;      // fixed anchors need no statistics
     if (p.C % 4 == 0)
         e = launch_pdl(k_frame_stats<4>, dim3(p.nsl), dim3(kNormThreads), st, (const float*)s.S, p.F, p.C, p.nsl,
                        s.Dp, s.Qp, s.Gp, s.hdr);

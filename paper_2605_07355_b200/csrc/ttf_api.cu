@@ -33,7 +33,7 @@ int sm_count() {
 }
 
 // ---- optional per-kernel timing: CUDA events recorded around every launch while profiling is on ---------
-enum { PK_NORM_ANCHOR = 0, PK_MATCH = 1, PK_COMPACT = 2, PK_FUSE_COUNT = 3, PK_KINDS = 4 };
+enum { PK_NORM_SUM = 0, PK_FRAME_STATS = 1, PK_MATCH = 2, PK_COMPACT = 3, PK_FUSE_COUNT = 4, PK_KINDS = 5 };
 struct ProfRecord { int kind; cudaEvent_t a, b; };
 static std::mutex g_prof_mu;
 static bool g_prof_on = false;
@@ -150,7 +150,12 @@ static int clear_control(const Problem&, void* ws, cudaStream_t st) {
 static int run_front(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                      unsigned char* keep, cudaStream_t st) {
     cudaError_t e;
-    { ProfScope ps(st, PK_NORM_ANCHOR); e = launch_norm_anchor(p, s, out_anchor, st); }
+    { ProfScope ps(st, PK_NORM_SUM); e = launch_norm_sum(p, s, st); }
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (p.anchor_mode == 0) {
+        ProfScope ps(st, PK_FRAME_STATS);
+        e = launch_frame_stats(p, s, out_anchor, st);
+    }
     if (e != cudaSuccess) return cuda_fail(e);
     { ProfScope ps(st, PK_MATCH); e = launch_match(p, s, out_anchor, shat, dst, keep, st); }
     if (e != cudaSuccess) return cuda_fail(e);

@@ -76,7 +76,8 @@ inline bool uses_mma_match(const Problem& p) {
 void carve_scratch(const Problem& p, void* base, Scratch* s);
 
 // Kernel launchers (each enqueues on `st` and returns the launch error, if any).
-cudaError_t launch_norm_anchor(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st);
+cudaError_t launch_norm_sum(const Problem& p, const Scratch& s, cudaStream_t st);
+cudaError_t launch_frame_stats(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st);
 cudaError_t launch_match(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                          unsigned char* keep, cudaStream_t st);
 cudaError_t launch_fuse_count(const Problem& p, const Scratch& s, const int* dst, const unsigned char* keep,
