@@ -178,7 +178,10 @@ __device__ __forceinline__ int select_in_frame(const unsigned char* __restrict__
 // Gather with bulk asynchronous copies, for rows that are 16-byte aligned multiples of 16 bytes: a warp finds the
 // source row of its output row as above, then one lane moves the row global -> shared -> global with two bulk
 // copies per piece of at most kBulkPiece bytes, so no data passes through registers.
-constexpr int kBulkPiece = 8192;
+#ifndef TTF_BULK_PIECE
+#define TTF_BULK_PIECE 8192
+#endif
+constexpr int kBulkPiece = TTF_BULK_PIECE;
 
 __global__ void __launch_bounds__(kCopyWarps * 32)
 k_compact_bulk(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, int W, int r,
