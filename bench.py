@@ -51,6 +51,12 @@ def parse_args():
     return ap.parse_args()
 
 
+# DRAM bytes (read + write) per launch from the committed ncu capture (profiles/kernels_full_vl8b_cal.md: cold
+# caches, one launch of each kernel).  Valid only for the kernels as captured; other workloads report null.
+NCU_TRAFFIC = {("vl8b_cal", "match"): 67274496 + 1014784, ("vl8b_cal", "norm_sum"): 67120128 + 324096,
+               ("vl8b_cal", "compact"): 24685568 + 58624}
+
+
 def peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -355,7 +361,9 @@ def main():
     kbytes = A.kernel_bytes(dominant, spec.F, spec.N, C, spec.itemsize, int(round(avg_count)))
     achieved = kbytes / (kern[dominant]["us_per_launch"] * 1e-6) / 1e9
     roofline = {"bound": "hbm", "kernel": dominant, "timed": "alone, single stream, CUDA events around each launch", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
-                "frac": achieved / peak_gbs, "peak_source": f"of {peak_kind}", "traffic": None,
+                "frac": achieved / peak_gbs, "peak_source": f"of {peak_kind}",
+                "traffic": NCU_TRAFFIC.get((spec.name, dominant)) if amode == 0 else None,
+                "traffic_note": "ncu, cold caches (in the pipeline the second pass over X is served by L2 when one clip is in flight)",
                 "algorithmic_bytes_per_launch": kbytes,
                 "kernel_share": {k: prof[k][0] / tot for k in kern},
                 "kernel_us": {k: round(kern[k]["us_per_launch"], 3) for k in kern}}
