@@ -128,6 +128,37 @@ int ttf_query_ex(const void* features, int F, int H, int W, int C, int r, float 
                  int* out_fuse_cnt, ttf_stream_t stream);
 
 /*
+ * Streaming segment (Discussion D3: the last frame of each segment serves as a rolling anchor; new frames are
+ * compressed against it and appended to the KV cache).  features = [F, H, W, C] whose frame 0 is the rolling
+ * anchor, i.e. the last frame of the previous segment, which the consumer already holds; frames 1..F-1 are the
+ * new ones and are matched against frame 0.  Only the preserved new tokens are emitted (no anchor rows):
+ * out_count = P, rows in ascending flat order, positions (frame_base + k - 1, y, x) so that frame 1 of the
+ * segment carries the video frame index frame_base.  Capacity (F-1)*H*W rows.  Otherwise as ttf_compress.
+ */
+int ttf_compress_segment(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                         int frame_base, void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream);
+
+/*
+ * TTF-R restoration (Discussion D4: a restoration step reconstructs the full spatio-temporal layout through
+ * the mapping dst(k,i), Eq. dst).  `compressed` holds one row of row_bytes bytes per token of the compressed
+ * sequence, in the order ttf_compress emits (any payload: the tokens themselves or what a model computed for
+ * them).  out_full [F*H*W rows] receives, for token (k,i), its own compressed row if it was retained, else the
+ * anchor row dst(k,i) it was fused into.  anchor (one device int), keep and dst are ttf_query's outputs.
+ * row_index [F*H*W] int32 is written with the source row of every token (scratch and result).
+ */
+int ttf_restore(const void* compressed, size_t row_bytes, int F, int H, int W, const int* anchor,
+                const unsigned char* keep, const int* dst, void* out_full, int* row_index, ttf_stream_t stream);
+
+/*
+ * The statistic an adaptive threshold would be calibrated on (Discussion D1: the empirical distribution of the
+ * best-match similarities of the current clip; the paper gives no rule for choosing t from it, so only the
+ * distribution is computed).  out_hist [bins] uint32: counts of best_sim over the source tokens (anchor frame
+ * excluded, NaN skipped) in `bins` equal bins of [-1, 1]: bin = floor((s + 1) / 2 * bins), clamped to the range.
+ */
+int ttf_sim_histogram(const float* best_sim, const int* anchor, int F, int H, int W, int bins,
+                      unsigned int* out_hist, ttf_stream_t stream);
+
+/*
  * The same pass for callers whose tensors live in HOST memory (all four pointers are host pointers; pinned
  * memory makes the copies asynchronous).  Copies features to the device, runs ttf_compress, copies L' and the
  * first L' rows of tokens and positions back, and returns after synchronising.  Device staging buffers are

@@ -218,5 +218,48 @@ int ttf_oracle_compact(const void* Xbytes, size_t row_bytes, const uint8_t* keep
     return L;
 }
 
+/*
+ * TTF-R restoration (Discussion D4): the row of the compressed sequence that stands for token (k,i) is its own
+ * row if m_{k,i} = 1 (anchor rows 0..N-1, then preserved source tokens in ascending flat order), else the anchor
+ * row dst(k,i).  Fills row_index[F*N] and, if out_full is given, copies the rows (row_bytes each).
+ */
+void ttf_oracle_restore(const void* compressed, size_t row_bytes, const uint8_t* keep, const int* dst,
+                        int F, int N, int a, int* row_index, void* out_full) {
+    int next = N;                                   /* next preserved source row */
+    for (int k = 0; k < F; ++k)
+        for (int i = 0; i < N; ++i) {
+            size_t f = (size_t)k * N + i;
+            int row;
+            if (k == a) row = i;
+            else if (keep[f]) row = next++;
+            else row = dst[f];
+            row_index[f] = row;
+            if (out_full)
+                memcpy((char*)out_full + f * row_bytes, (const char*)compressed + (size_t)row * row_bytes, row_bytes);
+        }
+}
+
+/*
+ * Distribution of the best-match similarities of the source tokens (Discussion D1): counts over `bins` equal
+ * bins of [-1, 1], bin = floor((s + 1) / 2 * bins) evaluated in fp32 like the CUDA path, clamped; NaN skipped.
+ */
+void ttf_oracle_sim_histogram(const float* s_hat, int F, int N, int a, int bins, unsigned int* hist) {
+    for (int b = 0; b < bins; ++b) hist[b] = 0;
+    for (int k = 0; k < F; ++k) {
+        if (k == a) continue;
+        for (int i = 0; i < N; ++i) {
+            float s = s_hat[(size_t)k * N + i];
+            if (!(s == s)) continue;
+            volatile float u = s + 1.0f;            /* keep every step in fp32 */
+            volatile float v = u * 0.5f;
+            volatile float x = v * (float)bins;
+            int b = (int)floorf(x);
+            if (b < 0) b = 0;
+            if (b >= bins) b = bins - 1;
+            hist[b] += 1;
+        }
+    }
+}
+
 /* Cache-aware Decode Alignment, Eqs. (Lpre), (decode_pos): pos_dec(l) = L' + T + l */
 long long ttf_oracle_decode_pos(long long L_prime, long long T, long long l) { return L_prime + T + l; }

@@ -47,6 +47,10 @@ def _load():
         lib.ttf_oracle_fuse_count.argtypes = [vp, vp, c_int, c_int, c_int, vp]
         lib.ttf_oracle_compact.restype = c_int
         lib.ttf_oracle_compact.argtypes = [vp, c_sz, vp, c_int, c_int, c_int, c_int, vp, vp, vp]
+        lib.ttf_oracle_restore.restype = None
+        lib.ttf_oracle_restore.argtypes = [vp, c_sz, vp, vp, c_int, c_int, c_int, vp, vp]
+        lib.ttf_oracle_sim_histogram.restype = None
+        lib.ttf_oracle_sim_histogram.argtypes = [vp, c_int, c_int, c_int, c_int, vp]
         lib.ttf_oracle_decode_pos.restype = ctypes.c_longlong
         lib.ttf_oracle_decode_pos.argtypes = [ctypes.c_longlong] * 3
         _lib = lib
@@ -137,6 +141,37 @@ def compact(X: np.ndarray, keep: np.ndarray, a: int):
     L = _load().ttf_oracle_compact(_ptr(Xc), C * X.dtype.itemsize, _ptr(keep), F, H, W, int(a),
                                    _ptr(tokens), _ptr(pos), _ptr(index))
     return tokens[:L], pos[:L], index[:L], int(L)
+
+
+def restore(compressed: np.ndarray, keep: np.ndarray, dst: np.ndarray, F: int, N: int, a: int):
+    """Discussion D4 (TTF-R): returns (full[F*N, ...], row_index[F*N])."""
+    comp = np.ascontiguousarray(compressed)
+    keep = np.ascontiguousarray(keep, dtype=np.uint8)
+    dst = np.ascontiguousarray(dst, dtype=np.int32)
+    row_bytes = comp[0].size * comp.itemsize
+    full = np.empty((F * N,) + comp.shape[1:], dtype=comp.dtype)
+    idx = np.empty(F * N, dtype=np.int32)
+    _load().ttf_oracle_restore(_ptr(comp), row_bytes, _ptr(keep), _ptr(dst), F, N, int(a), _ptr(idx), _ptr(full))
+    return full, idx
+
+
+def sim_histogram(s_hat_f32: np.ndarray, F: int, N: int, a: int, bins: int) -> np.ndarray:
+    """Discussion D1: histogram of the best similarities of the source tokens over [-1, 1]."""
+    s = np.ascontiguousarray(s_hat_f32, dtype=np.float32)
+    hist = np.empty(bins, dtype=np.uint32)
+    _load().ttf_oracle_sim_histogram(_ptr(s), F, N, int(a), int(bins), _ptr(hist))
+    return hist
+
+
+def compress_segment(X: np.ndarray, r: int, t: float, frame_base: int, forced_keep: Optional[np.ndarray] = None):
+    """Discussion D3 (rolling anchor): frame 0 is the anchor of the segment and is not emitted; returns
+    (tokens[P, C], pos[P, 3] with the frame coordinate frame_base + k - 1, P)."""
+    F, H, W, C = _shape(X)
+    N = H * W
+    R = compress(X, r, t, anchor_frame=0, forced_keep=forced_keep)
+    pos = R.pos[N:].copy()
+    pos[:, 0] += frame_base - 1
+    return R.tokens[N:], pos, R.count - N
 
 
 def decode_pos(L_prime: int, T: int, l: int) -> int:

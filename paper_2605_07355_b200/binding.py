@@ -21,7 +21,8 @@ TTF_OK = 0
 EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
-    "ttf_query_static", "ttf_compress_ex", "ttf_query_ex",
+    "ttf_query_static", "ttf_compress_ex", "ttf_query_ex", "ttf_compress_segment", "ttf_restore",
+    "ttf_sim_histogram",
 ]
 TTF_ANCHOR_AUTO, TTF_ANCHOR_FIRST, TTF_ANCHOR_LAST, TTF_ANCHOR_EXPLICIT = 0, 1, 2, 3
 TTF_STATIC_SCRATCH_BYTES = 8 << 20
@@ -66,6 +67,12 @@ def lib() -> ctypes.CDLL:
         L.ttf_compress_ex.argtypes = [vp] + shape + [f, i, i, i, vp, vp, vp, vp]
         L.ttf_query_ex.restype = i
         L.ttf_query_ex.argtypes = [vp] + shape + [f, i, i, i, vp, vp, vp, vp, vp, vp]
+        L.ttf_compress_segment.restype = i
+        L.ttf_compress_segment.argtypes = [vp] + shape + [f, i, i, vp, vp, vp, vp]
+        L.ttf_restore.restype = i
+        L.ttf_restore.argtypes = [vp, sz, i, i, i, vp, vp, vp, vp, vp, vp]
+        L.ttf_sim_histogram.restype = i
+        L.ttf_sim_histogram.argtypes = [vp, vp, i, i, i, i, vp, vp]
         L.ttf_query_static.restype = i
         L.ttf_query_static.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp]
         L.ttf_compress_host.restype = i
@@ -199,6 +206,51 @@ def ttf_query_static(features: torch.Tensor, r: int, t: float, out: dict, stream
     if rc != TTF_OK:
         raise TTFError(rc, "ttf_query_static")
     return out
+
+
+def ttf_compress_segment(features: torch.Tensor, r: int, t: float, frame_base: int, stream=None):
+    """ttf_compress_segment: frame 0 is the rolling anchor, frames 1.. are compressed against it; returns
+    (out_tokens [(F-1)*H*W, C], out_count int32[1] = P, out_pos_thw [(F-1)*H*W, 3])."""
+    F, H, W, C = _check_features(features, "cuda")
+    dev = features.device
+    n = max(1, (F - 1) * H * W)
+    out_tokens = torch.empty((n, C), dtype=features.dtype, device=dev)
+    out_count = torch.empty(1, dtype=torch.int32, device=dev)
+    out_pos = torch.empty((n, 3), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ttf_compress_segment(_p(features), F, H, W, C, int(r), float(t), _dtype_code(features),
+                                        int(frame_base), _p(out_tokens), _p(out_count), _p(out_pos), _stream_ptr(stream))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_compress_segment")
+    return out_tokens, out_count, out_pos
+
+
+def ttf_restore(compressed: torch.Tensor, F: int, H: int, W: int, anchor: torch.Tensor, keep: torch.Tensor,
+                dst: torch.Tensor, stream=None):
+    """ttf_restore: returns (out_full [F*H*W, ...row shape], row_index int32 [F*H*W])."""
+    if not compressed.is_contiguous():
+        raise ValueError("compressed must be contiguous")
+    dev = compressed.device
+    row_bytes = compressed[0].numel() * compressed.element_size()
+    out = torch.empty((F * H * W,) + tuple(compressed.shape[1:]), dtype=compressed.dtype, device=dev)
+    idx = torch.empty(F * H * W, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ttf_restore(_p(compressed), row_bytes, F, H, W, _p(anchor), _p(keep), _p(dst), _p(out), _p(idx),
+                               _stream_ptr(stream))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_restore")
+    return out, idx
+
+
+def ttf_sim_histogram(best_sim: torch.Tensor, anchor: torch.Tensor, F: int, H: int, W: int, bins: int, stream=None):
+    """ttf_sim_histogram: uint32 counts [bins] (returned as an int32 tensor with the same bits)."""
+    dev = best_sim.device
+    hist = torch.empty(bins, dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ttf_sim_histogram(_p(best_sim), _p(anchor), F, H, W, int(bins), _p(hist), _stream_ptr(stream))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_sim_histogram")
+    return hist
 
 
 def ttf_compress_host(features: torch.Tensor, r: int, t: float, out_tokens: Optional[torch.Tensor] = None,

@@ -99,7 +99,7 @@ static int make_problem(const void* X, int F, int H, int W, int C, int r, float 
     p->nslice = p->nq * (p->ls / 32);
     if ((long long)F * p->nq >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
     p->nsl = C % 4 == 0 ? (C + 127) / 128 : (C + 31) / 32;
-    p->anchor_mode = 0; p->anchor_arg = 0;
+    p->anchor_mode = 0; p->anchor_arg = 0; p->emit_anchor = 1; p->pos_t_offset = 0;
     return TTF_OK;
 }
 
@@ -372,6 +372,41 @@ int ttf_query_ex(const void* features, int F, int H, int W, int C, int r, float 
     rc = cached_scratch(s.bytes, (cudaStream_t)stream, &ws);
     if (rc != TTF_OK) return rc;
     return query_impl(p, ws, out_anchor, out_keep, out_dst, out_best_sim, out_fuse_cnt, (cudaStream_t)stream);
+}
+
+int ttf_compress_segment(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                         int frame_base, void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream) {
+    if (!features || !out_tokens || !out_count || !out_pos_thw) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
+    if (rc == TTF_OK) rc = set_anchor_rule(&p, TTF_ANCHOR_FIRST, 0);
+    if (rc != TTF_OK) return rc;
+    p.emit_anchor = 0;
+    p.pos_t_offset = frame_base - 1;             // frame 1 of the segment is frame `frame_base` of the video
+    Scratch s;
+    carve_scratch(p, nullptr, &s);
+    void* ws = nullptr;
+    rc = cached_scratch(s.bytes, (cudaStream_t)stream, &ws);
+    if (rc != TTF_OK) return rc;
+    return compress_impl(p, ws, out_tokens, out_count, out_pos_thw, (cudaStream_t)stream);
+}
+
+int ttf_restore(const void* compressed, size_t row_bytes, int F, int H, int W, const int* anchor,
+                const unsigned char* keep, const int* dst, void* out_full, int* row_index, ttf_stream_t stream) {
+    if (!compressed || !anchor || !keep || !dst || !out_full || !row_index) return TTF_ERR_INVALID_ARG;
+    if (F < 1 || H < 1 || W < 1 || row_bytes < 1) return TTF_ERR_INVALID_ARG;
+    if ((long long)F * H * W >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
+    cudaError_t e = launch_restore(compressed, row_bytes, F, H * W, anchor, keep, dst, out_full, row_index,
+                                   (cudaStream_t)stream);
+    return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+}
+
+int ttf_sim_histogram(const float* best_sim, const int* anchor, int F, int H, int W, int bins,
+                      unsigned int* out_hist, ttf_stream_t stream) {
+    if (!best_sim || !anchor || !out_hist || F < 1 || H < 1 || W < 1 || bins < 1) return TTF_ERR_INVALID_ARG;
+    if ((long long)F * H * W >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
+    cudaError_t e = launch_sim_histogram(best_sim, anchor, F, H * W, bins, out_hist, (cudaStream_t)stream);
+    return e == cudaSuccess ? TTF_OK : cuda_fail(e);
 }
 
 int ttf_query_static(const void* features, int F, int H, int W, int C, int r, float t, int dtype,

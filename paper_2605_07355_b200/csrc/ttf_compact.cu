@@ -188,7 +188,7 @@ k_compact_bulk(const unsigned char* __restrict__ X, size_t row_bytes, int F, int
                const int* __restrict__ hdr, const int* __restrict__ cnt, const int* __restrict__ gprefix,
                const unsigned char* __restrict__ keep, const int* __restrict__ dst,
                unsigned char* __restrict__ out_tokens, int* __restrict__ out_pos, int* __restrict__ out_count,
-               int* __restrict__ fuse_cnt, int ncopy_blocks)
+               int* __restrict__ fuse_cnt, int ncopy_blocks, int NA, int t_off)
 {
     extern __shared__ __align__(128) unsigned char stage[];     // [kCopyWarps][kBulkPiece]
     __shared__ uint64_t bar[kCopyWarps];
@@ -210,7 +210,7 @@ k_compact_bulk(const unsigned char* __restrict__ X, size_t row_bytes, int F, int
     if (gw == 0) {                               // L' = N + P (Eq. Lpre)
         int kk, bb;
         const int P = find_frame(cnt, gprefix, F, a, lane, -1, kk, bb);
-        if (lane == 0) *out_count = __ldcg(hdr + HDR_ERROR) ? -1 : N + P;
+        if (lane == 0) *out_count = __ldcg(hdr + HDR_ERROR) ? -1 : NA + P;
     }
     unsigned char* buf = stage + (size_t)w * kBulkPiece;
     const int pieces = (int)((row_bytes + kBulkPiece - 1) / kBulkPiece);
@@ -218,18 +218,18 @@ k_compact_bulk(const unsigned char* __restrict__ X, size_t row_bytes, int F, int
     bool gave_up = false;
     for (int j = gw; ; j += nw) {
         int f;
-        if (j < N) f = a * N + j;                // anchor rows first (Eq. xprime_stack)
+        if (j < NA) f = a * N + j;               // anchor rows first (Eq. xprime_stack)
         else {
             int k, before;
-            find_frame(cnt, gprefix, F, a, lane, j - N, k, before);
+            find_frame(cnt, gprefix, F, a, lane, j - NA, k, before);
             if (k < 0) break;                    // past the last output row
-            const int i = select_in_frame(keep + (size_t)k * N, N, j - N - before, lane);
+            const int i = select_in_frame(keep + (size_t)k * N, N, j - NA - before, lane);
             if (i < 0) break;                    // cannot happen when cnt matches keep
             f = k * N + i;
         }
         if (lane < 3) {                          // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
             const int k = f / N, i = f - k * N, yy = i / W;
-            out_pos[(size_t)j * 3 + lane] = lane == 0 ? k : (lane == 1 ? yy : i - yy * W);
+            out_pos[(size_t)j * 3 + lane] = lane == 0 ? k + t_off : (lane == 1 ? yy : i - yy * W);
         }
         if (lane == 0 && !gave_up) {
             for (int pc = 0; pc < pieces; ++pc) {
@@ -259,7 +259,7 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
           const int* __restrict__ hdr, const int* __restrict__ cnt, const int* __restrict__ gprefix,
           const unsigned char* __restrict__ keep, const int* __restrict__ dst,
           unsigned char* __restrict__ out_tokens, int* __restrict__ out_pos, int* __restrict__ out_count,
-          int* __restrict__ fuse_cnt, int ncopy_blocks)
+          int* __restrict__ fuse_cnt, int ncopy_blocks, int NA, int t_off)
 {
     using U = typename CopyUnit<COPY_BYTES>::type;
     const int N = H * W;
@@ -285,23 +285,23 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
         int kk, bb;
         const int P = find_frame(cnt, gprefix, F, a, lane, -1, kk, bb);
         // a bounded wait of an earlier kernel of this call gave up: report instead of a plausible count
-        if (lane == 0) *out_count = __ldcg(hdr + HDR_ERROR) ? -1 : N + P;
+        if (lane == 0) *out_count = __ldcg(hdr + HDR_ERROR) ? -1 : NA + P;
     }
     const int upr = (int)(row_bytes / COPY_BYTES);         // copy units per row
     for (int j = gw; ; j += nw) {
         int f;
-        if (j < N) f = a * N + j;                          // anchor rows first (Eq. xprime_stack)
+        if (j < NA) f = a * N + j;                         // anchor rows first (Eq. xprime_stack)
         else {
             int k, before;
-            find_frame(cnt, gprefix, F, a, lane, j - N, k, before);
+            find_frame(cnt, gprefix, F, a, lane, j - NA, k, before);
             if (k < 0) break;                              // past the last output row
-            const int i = select_in_frame(keep + (size_t)k * N, N, j - N - before, lane);
+            const int i = select_in_frame(keep + (size_t)k * N, N, j - NA - before, lane);
             if (i < 0) break;                              // cannot happen when cnt matches keep
             f = k * N + i;
         }
         if (lane < 3) {                                    // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
             const int k = f / N, i = f - k * N, yy = i / W;
-            out_pos[(size_t)j * 3 + lane] = lane == 0 ? k : (lane == 1 ? yy : i - yy * W);
+            out_pos[(size_t)j * 3 + lane] = lane == 0 ? k + t_off : (lane == 1 ? yy : i - yy * W);
         }
         const U* src = reinterpret_cast<const U*>(X + (size_t)f * row_bytes);
         U* dsto = reinterpret_cast<U*>(out_tokens + (size_t)j * row_bytes);
@@ -322,7 +322,7 @@ cudaError_t launch_fuse_count(const Problem& p, const Scratch& s, const int* dst
     const int nb = (p.N + kCopyWarps - 1) / kCopyWarps;
     k_compact<4><<<nb < 1024 ? nb : 1024, kCopyWarps * 32, 0, st>>>(
         nullptr, 0, p.F, p.H, p.W, p.r, s.hdr, s.cnt, s.prefix, keep, dst, nullptr, nullptr, nullptr,
-        fuse_cnt, 0);
+        fuse_cnt, 0, p.N, 0);
     return cudaGetLastError();
 }
 
@@ -345,6 +345,7 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
     const unsigned char* X = reinterpret_cast<const unsigned char*>(p.X);
     unsigned char* out = reinterpret_cast<unsigned char*>(out_tokens);
     const dim3 g(grid), b(kCopyWarps * 32);
+    const int NA = p.emit_anchor ? p.N : 0;      // a streaming segment does not emit its rolling anchor again
     // the pre-scanned prefix of very long clips is read through plain loads: order that case by the stream
     const bool pdl = p.F <= kWarpPrefixMaxF;
     if (vec) {
@@ -363,15 +364,15 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
         cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
         return cudaLaunchKernelEx(&cfg, k_compact_bulk, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
                                   (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep,
-                                  (const int*)s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy);
+                                  (const int*)s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy, NA, p.pos_t_offset);
     }
     if (esize == 4)
         return launch_pdl_if(pdl, k_compact<4>, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
                           (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep, (const int*)s.dst,
-                          out, out_pos, out_count, s.fuse_cnt, ncopy);
+                          out, out_pos, out_count, s.fuse_cnt, ncopy, NA, p.pos_t_offset);
     return launch_pdl_if(pdl, k_compact<2>, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
                       (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep, (const int*)s.dst,
-                      out, out_pos, out_count, s.fuse_cnt, ncopy);
+                      out, out_pos, out_count, s.fuse_cnt, ncopy, NA, p.pos_t_offset);
 }
 
 }  // namespace ttf

@@ -33,6 +33,8 @@ struct Problem {
     int nsl;            // frame statistics: channel slices (128 channels when C % 4 == 0, else 32)
     int anchor_mode;    // 0 auto (Eq. auto_anchor), 1 first, 2 last, 3 explicit
     int anchor_arg;     // explicit anchor frame
+    int emit_anchor;    // 1: X' starts with the N anchor rows (Eq. xprime_stack); 0: streaming segment, sources only
+    int pos_t_offset;   // added to the frame coordinate of every emitted position
 };
 
 // Device pointers carved out of one scratch allocation.
@@ -84,6 +86,12 @@ cudaError_t launch_fuse_count(const Problem& p, const Scratch& s, const int* dst
                               int* fuse_cnt, cudaStream_t st);
 cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens, int* out_pos, int* out_count,
                            cudaStream_t st);
+
+cudaError_t launch_restore(const void* comp, size_t row_bytes, int F, int N, const int* anchor,
+                           const unsigned char* keep, const int* dst, void* out_full, int* row_index,
+                           cudaStream_t st);
+cudaError_t launch_sim_histogram(const float* sim, const int* anchor, int F, int N, int bins, unsigned int* hist,
+                                 cudaStream_t st);
 
 int sm_count();   // SMs of the current device (cached per device)
 

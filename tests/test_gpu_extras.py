@@ -1,0 +1,70 @@
+"""GPU parity of the extensions from the paper's Discussion: streaming segment (D3), TTF-R restoration (D4) and
+the best-similarity histogram (D1), each against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ttf_oracle as O
+from paper_2605_07355_b200 import clips
+import paper_2605_07355_b200 as P
+from tests.parity import to_device, to_bits
+from tests.test_gpu_parity import corr_clip
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("shape,dtype", [((4, 6, 5, 64), "bf16"), ((5, 3, 7, 40), "f32"), ((3, 4, 4, 33), "bf16"),
+                                         ((32, 16, 16, 256), "bf16")])
+def test_restore_matches_oracle(shape, dtype):
+    F, H, W, C = shape
+    N = H * W
+    X = corr_clip(F, H, W, C, seed=91 + C, dtype=dtype)
+    Xd = to_device(X)
+    q = P.ttf_query(Xd, 1, 0.7)
+    toks, cnt, pos = P.ttf_compress(Xd, 1, 0.7)
+    torch.cuda.synchronize()
+    L = int(cnt.item())
+    full, idx = P.ttf_restore(toks[:L].contiguous(), F, H, W, q["anchor"], q["keep"], q["dst"])
+    torch.cuda.synchronize()
+    keep, dst, a = q["keep"].cpu().numpy(), q["dst"].cpu().numpy(), int(q["anchor"].item())
+    ref_full, ref_idx = O.restore(to_bits(toks[:L]), keep, dst, F, N, a)
+    assert (idx.cpu().numpy() == ref_idx).all()
+    assert (to_bits(full) == ref_full).all()
+    Xf = X.reshape(F * N, C)
+    assert (to_bits(full)[keep.astype(bool)] == Xf[keep.astype(bool)]).all()
+    # a payload that is not the tokens (e.g. hidden states), odd row size
+    payload = torch.arange(L * 3, dtype=torch.float32, device="cuda").reshape(L, 3)
+    full2, _ = P.ttf_restore(payload, F, H, W, q["anchor"], q["keep"], q["dst"])
+    assert (full2.cpu().numpy() == payload.cpu().numpy()[ref_idx]).all()
+
+
+@pytest.mark.parametrize("bins", [1, 16, 100])
+def test_histogram_matches_oracle(bins):
+    s = clips.CONFIGS["vl2b_cal"]
+    Xd = to_device(clips.make_clip(s))
+    q = P.ttf_query(Xd, s.r, s.t)
+    hist = P.ttf_sim_histogram(q["best_sim"], q["anchor"], s.F, s.H, s.W, bins)
+    torch.cuda.synchronize()
+    ref = O.sim_histogram(q["best_sim"].cpu().numpy(), s.F, s.N, int(q["anchor"].item()), bins)
+    got = hist.cpu().numpy().view(np.uint32)
+    assert (got == ref).all() and got.sum() == (s.F - 1) * s.N
+
+
+@pytest.mark.parametrize("shape,dtype", [((4, 6, 5, 64), "bf16"), ((5, 3, 7, 40), "f32"), ((9, 16, 16, 512), "bf16")])
+def test_segment_matches_oracle(shape, dtype):
+    F, H, W, C = shape
+    N = H * W
+    X = corr_clip(F, H, W, C, seed=95 + C, dtype=dtype)
+    Xd = to_device(X)
+    toks, cnt, pos = P.ttf_compress_segment(Xd, 1, 0.7, frame_base=17)
+    q = P.ttf_query(Xd, 1, 0.7, anchor_mode=P.TTF_ANCHOR_FIRST)
+    torch.cuda.synchronize()
+    keep = q["keep"].cpu().numpy()
+    R = O.compress(X, 1, 0.7, anchor_frame=0)
+    in_band = np.abs(R.s_hat.astype(np.float32) - np.float32(0.7)) < 1e-4
+    assert not ((keep != R.keep) & ~in_band).any()
+    ref_t, ref_p, ref_P = O.compress_segment(X, 1, 0.7, 17, forced_keep=keep)
+    Pn = int(cnt.item())
+    assert Pn == ref_P == int(keep.sum()) - N
+    assert (pos[:Pn].cpu().numpy() == ref_p).all() and (to_bits(toks[:Pn]) == ref_t).all()
+    assert Pn == 0 or int(pos[:Pn, 0].min().item()) >= 17

@@ -264,3 +264,61 @@ def test_bf16_bits_equal_their_fp32_widening():
 def test_decode_alignment():
     assert O.decode_pos(2703, 57, 0) == 2703 + 57
     assert O.decode_pos(2703, 57, 9) == 2703 + 57 + 9
+
+
+# ---- Discussion D4: restoration through dst ----------------------------------------------------------------
+def test_restore_inverts_compaction():
+    F, H, W, C = 4, 5, 4, 16
+    N = H * W
+    X = corr_clip(F, H, W, C, seed=81)
+    R = O.compress(X, 1, 0.70)
+    full, idx = O.restore(R.tokens, R.keep, R.dst, F, N, R.anchor)
+    Xf = X.reshape(F * N, C)
+    kept = R.keep.astype(bool)
+    assert (full[kept] == Xf[kept]).all()                               # retained tokens come back unchanged
+    fused = np.flatnonzero(~kept)
+    assert (full[fused] == Xf[R.anchor * N + R.dst[fused]]).all()       # fused ones become their anchor match
+    assert (idx[fused] == R.dst[fused]).all() and (idx[R.anchor * N:(R.anchor + 1) * N] == np.arange(N)).all()
+    assert sorted(idx[kept].tolist()) == list(range(R.count))           # a bijection onto the compressed rows
+    # nothing fused: restoration is the identity
+    R2 = O.compress(X, 1, 1.5)
+    full2, idx2 = O.restore(R2.tokens, R2.keep, R2.dst, F, N, R2.anchor)
+    assert (full2 == Xf).all()
+    # everything fused with identical frames: every frame becomes the anchor frame
+    Xi = np.repeat(X[:1], 3, axis=0)
+    R3 = O.compress(Xi, 1, 0.7)
+    full3, _ = O.restore(R3.tokens, R3.keep, R3.dst, 3, N, R3.anchor)
+    assert (full3.reshape(3, N, C) == Xi.reshape(3, N, C)).all()
+
+
+# ---- Discussion D1: distribution of the best similarities ---------------------------------------------------
+@pytest.mark.parametrize("bins", [1, 7, 64, 200])
+def test_sim_histogram_matches_numpy(bins):
+    F, H, W, C = 5, 6, 5, 24
+    N = H * W
+    X = corr_clip(F, H, W, C, seed=83)
+    R = O.compress(X, 1, 0.70)
+    s = R.s_hat.astype(np.float32)
+    h = O.sim_histogram(s, F, N, R.anchor, bins)
+    src = np.delete(s.reshape(F, N), R.anchor, axis=0).ravel()
+    ref, _ = np.histogram(src.astype(np.float64), bins=bins, range=(-1.0, 1.0))
+    assert h.sum() == (F - 1) * N
+    # numpy bins in float64 with a closed last bin; values on a bin edge may land one bin apart
+    assert np.abs(h.astype(np.int64) - ref).sum() <= 2 and (h.astype(np.int64) == ref).mean() > 0.9
+    s2 = s.copy(); s2[N * ((R.anchor + 1) % F)] = np.nan
+    assert O.sim_histogram(s2, F, N, R.anchor, bins).sum() == (F - 1) * N - 1
+
+
+# ---- Discussion D3: streaming segment with a rolling anchor ---------------------------------------------------
+def test_segment_emits_only_new_preserved_tokens():
+    F, H, W, C = 4, 4, 5, 16
+    N = H * W
+    X = corr_clip(F, H, W, C, seed=85)
+    toks, pos, P = O.compress_segment(X, 1, 0.70, frame_base=9)
+    R = O.compress(X, 1, 0.70, anchor_frame=0)
+    assert P == R.count - N and (toks == R.tokens[N:]).all()
+    assert (pos[:, 0] == R.pos[N:, 0] + 8).all() and (pos[:, 1:] == R.pos[N:, 1:]).all()
+    assert pos[:, 0].min() >= 9                                          # frame 1 of the segment is video frame 9
+    t_all, p_all, P_all = O.compress_segment(X, 1, 1.5, frame_base=0)    # nothing fused: all new frames, in order
+    assert P_all == (F - 1) * N and (t_all == X[1:].reshape(-1, C)).all()
+    assert O.compress_segment(np.repeat(X[:1], 3, axis=0), 1, 0.7, 5)[2] == 0
