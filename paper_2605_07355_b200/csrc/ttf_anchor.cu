@@ -147,7 +147,7 @@ static cudaError_t launch_sum_t(const Problem& p, const Scratch& s, cudaStream_t
     const T* X = reinterpret_cast<const T*>(p.X);
     const unsigned blocks = (unsigned)((long long)p.F * p.nq);
     const dim3 g(blocks), b(kNormThreads);
-    if (uses_mma_match(p))
+    if (!needs_sweep_norms(p))
         return launch_pdl(k_norm_sum<T, V, 32, false>, g, b, st, X, p.F, p.N, p.C, p.nq, s.S, s.ssq, s.cnt, s.hdr);
     return launch_pdl(k_norm_sum<T, V, 32, true>, g, b, st, X, p.F, p.N, p.C, p.nq, s.S, s.ssq, s.cnt, s.hdr);
 }

@@ -74,6 +74,9 @@ inline bool uses_mma_match(const Problem& p) {
     return p.dtype == 1 && p.vec && p.r <= 2 && (long long)p.N * ((p.F + 15) / 16) < (1LL << 31);
 }
 
+// The sweep stores per-token partial squared norms only for the kernels that read them.
+inline bool needs_sweep_norms(const Problem& p) { return !uses_mma_match(p) || p.r == 2; }
+
 // Fills the offsets (base may be NULL to only compute `bytes`).
 void carve_scratch(const Problem& p, void* base, Scratch* s);
 

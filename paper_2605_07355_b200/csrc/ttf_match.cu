@@ -119,17 +119,11 @@ constexpr int kMmaWarps = 8;
 #ifndef TTF_MMA_MAXREG
 #define TTF_MMA_MAXREG 96
 #endif
-constexpr int kMmaStages = TTF_MMA_STAGES;       // cp.async stages per warp (kMmaStages - 1 blocks in flight)
+constexpr int kMmaStagesDefault = TTF_MMA_STAGES; // cp.async stages per warp (stages - 1 blocks in flight)
 
 // One pipeline stage of a warp: the 16-byte fragment pieces of its 64-byte block, (2 MT + NT) per lane.  The
 // pieces travel global -> shared with cp.async (no registers are tied up while they are in flight, so a warp
 // keeps several stages outstanding); every lane copies into and later reads back its own 16-byte slots.
-template <int MT, int NT>
-struct MmaStage {
-    uint4 a[MT][2];
-    uint4 b[NT];
-};
-
 __device__ __forceinline__ void cp_async16(void* dst_smem, const void* src, bool valid) {
     const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(dst_smem));
     const int bytes = valid ? 16 : 0;            // 0 source bytes: the 16 destination bytes are zero-filled
@@ -153,55 +147,54 @@ __device__ __forceinline__ void mma_issue_stage(uint4* slot, const uint4* const 
     for (int nt = 0; nt < NT; ++nt) cp_async16(slot + (2 * MT + nt) * 32 + lane, brow[nt] + safe, ok && bvalid[nt]);
 }
 
-template <int MT, int NT>
-__device__ __forceinline__ void mma_read_stage(MmaStage<MT, NT>& sg, const uint4* slot, int lane) {
+// Consumes one landed stage of a warp: dot products of every source row with every candidate row and, when
+// GRAM, the squared norms of all rows: the Gram tile of a 16-row tile with itself has the squared norms on its
+// diagonal, so two extra MMAs per tile (columns = rows 0..7, then rows 8..15) give them on the tensor pipe from
+// fragments that are in registers anyway.  Fragments are read from the lane's slots tile by tile.
+template <int MT, int NT, bool GRAM>
+__device__ __forceinline__ void mma_consume_stage(const uint4* slot, int lane, float (&acc)[MT][NT][4],
+                                                  float (&accn)[GRAM ? MT : 1][2][4], float (&accb)[GRAM ? NT : 1][4]) {
+    uint4 b[NT];
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-        for (int h = 0; h < 2; ++h) sg.a[mt][h] = slot[(mt * 2 + h) * 32 + lane];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) sg.b[nt] = slot[(2 * MT + nt) * 32 + lane];
-}
-
-// Dot products of the stage, plus the squared norms of all its rows: the Gram tile of a 16-row tile with
-// itself has the squared norms on its diagonal, so two extra MMAs per tile (columns = rows 0..7, then rows
-// 8..15) give them on the tensor pipe from the fragments that are in registers anyway.
-template <int MT, int NT>
-__device__ __forceinline__ void mma_compute_stage(const MmaStage<MT, NT>& sg, float (&acc)[MT][NT][4],
-                                                  float (&accn)[MT][2][4], float (&accb)[NT][4]) {
+    for (int nt = 0; nt < NT; ++nt) b[nt] = slot[(2 * MT + nt) * 32 + lane];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
+        const uint4 a0 = slot[(mt * 2 + 0) * 32 + lane], a1 = slot[(mt * 2 + 1) * 32 + lane];
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
-            mma_bf16_16816(acc[mt][nt], sg.a[mt][0].x, sg.a[mt][1].x, sg.a[mt][0].y, sg.a[mt][1].y, sg.b[nt].x, sg.b[nt].y);
-            mma_bf16_16816(acc[mt][nt], sg.a[mt][0].z, sg.a[mt][1].z, sg.a[mt][0].w, sg.a[mt][1].w, sg.b[nt].z, sg.b[nt].w);
+            mma_bf16_16816(acc[mt][nt], a0.x, a1.x, a0.y, a1.y, b[nt].x, b[nt].y);
+            mma_bf16_16816(acc[mt][nt], a0.z, a1.z, a0.w, a1.w, b[nt].z, b[nt].w);
         }
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            mma_bf16_16816(accn[mt][h], sg.a[mt][0].x, sg.a[mt][1].x, sg.a[mt][0].y, sg.a[mt][1].y, sg.a[mt][h].x, sg.a[mt][h].y);
-            mma_bf16_16816(accn[mt][h], sg.a[mt][0].z, sg.a[mt][1].z, sg.a[mt][0].w, sg.a[mt][1].w, sg.a[mt][h].z, sg.a[mt][h].w);
+        if constexpr (GRAM) {
+            mma_bf16_16816(accn[mt][0], a0.x, a1.x, a0.y, a1.y, a0.x, a0.y);
+            mma_bf16_16816(accn[mt][0], a0.z, a1.z, a0.w, a1.w, a0.z, a0.w);
+            mma_bf16_16816(accn[mt][1], a0.x, a1.x, a0.y, a1.y, a1.x, a1.y);
+            mma_bf16_16816(accn[mt][1], a0.z, a1.z, a0.w, a1.w, a1.z, a1.w);
         }
     }
-    // candidate rows: rows of the Gram tile = slots of the tile pair (even, odd), columns = slots of tile nt
+    if constexpr (GRAM) {
+        // candidate rows: rows of the Gram tile = slots of the tile pair (even, odd), columns = slots of tile nt
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-        const uint4 lo = sg.b[nt & ~1];
-        const uint4 hi = (nt | 1) < NT ? sg.b[(nt | 1) < NT ? (nt | 1) : nt] : make_uint4(0, 0, 0, 0);
-        mma_bf16_16816(accb[nt], lo.x, hi.x, lo.y, hi.y, sg.b[nt].x, sg.b[nt].y);
-        mma_bf16_16816(accb[nt], lo.z, hi.z, lo.w, hi.w, sg.b[nt].z, sg.b[nt].w);
+        for (int nt = 0; nt < NT; ++nt) {
+            const uint4 lo = b[nt & ~1];
+            const uint4 hi = (nt | 1) < NT ? b[(nt | 1) < NT ? (nt | 1) : nt] : make_uint4(0, 0, 0, 0);
+            mma_bf16_16816(accb[nt], lo.x, hi.x, lo.y, hi.y, b[nt].x, b[nt].y);
+            mma_bf16_16816(accb[nt], lo.z, hi.z, lo.w, hi.w, b[nt].z, b[nt].w);
+        }
     }
 }
 
 // 96 registers and 3 stages (74 KB) per CTA: two of these CTAs leave room on an SM for a CTA of the next clip's
 // sweep, which is what lets clips on different streams overlap (measured: 31.6 vs 33.3 us per clip, 4 streams)
 #define TTF_MMA_BOUNDS __maxnreg__(TTF_MMA_MAXREG)
-template <int MT, int NT>
-__global__ void TTF_MMA_BOUNDS
-k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t,
-            AnchorSrc asrc,
-            float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep,
-            int* __restrict__ cnt)
+// GRAM: token norms from Gram-diagonal MMAs (else from the sweep's partial squared norms); ST: cp.async stages.
+template <int MT, int NT, bool GRAM, int ST>
+__device__ __forceinline__ void match_mma_body(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t,
+                                               const AnchorSrc& asrc, const float* ssq, int nslice,
+                                               float* __restrict__ shat, int* __restrict__ dst,
+                                               unsigned char* __restrict__ keep, int* __restrict__ cnt)
 {
+    constexpr int kMmaStages = ST;
     constexpr int FR = 16 * MT;      // frames per CTA
     constexpr int NC = 8 * NT;       // candidate slots per CTA (>= (2r+1)^2)
     constexpr int PIECES = 2 * MT + NT;
@@ -212,8 +205,8 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
     static_assert(sizeof(float) * kMmaWarps * FR * NC <= sizeof(uint4) * kMmaWarps * kMmaStages * PIECES * 32,
                   "partial products must fit the ring");
     __shared__ float s_dot[FR][NC];
-    __shared__ float s_na[kMmaWarps][FR];        // partial squared norms of the source rows, per warp
-    __shared__ float s_nb[kMmaWarps][NC];        // ... of the candidate rows
+    __shared__ float s_na[GRAM ? kMmaWarps : 1][FR];   // partial squared norms of the source rows, per warp
+    __shared__ float s_nb[GRAM ? kMmaWarps : 1][NC];   // ... of the candidate rows
     __shared__ float s_rs[FR];
     __shared__ float s_ra[NC];
     __shared__ int s_j[NC];
@@ -252,6 +245,13 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
     };
 
     if (tid < NC) s_j[tid] = cand_index(tid);
+    if constexpr (!GRAM) {                       // inverse norms from the sweep's partials
+        const size_t FN = (size_t)F * N;
+        for (int q = tid; q < FR + NC; q += kMmaWarps * 32) {
+            if (q < FR) { const int k = k0 + q; s_rs[q] = k < F ? inv_norm(ssq, nslice, FN, (size_t)k * N + i) : 0.f; }
+            else { const int j = cand_index(q - FR); s_ra[q - FR] = j >= 0 ? inv_norm(ssq, nslice, FN, (size_t)a * N + j) : 0.f; }
+        }
+    }
 
     const uint4* arow[MT][2];
 #pragma unroll
@@ -270,17 +270,17 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
         brow[nt] = reinterpret_cast<const uint4*>(X + ((size_t)a * N + (j >= 0 ? j : 0)) * C);
     }
 
-    float acc[MT][NT][4], accn[MT][2][4], accb[NT][4];
+    float acc[MT][NT][4], accn[GRAM ? MT : 1][2][4], accb[GRAM ? NT : 1][4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt) {
+        for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) acc[mt][nt][q] = 0.f;
-            accn[mt][0][q] = 0.f; accn[mt][1][q] = 0.f;
-        }
 #pragma unroll
-        for (int nt = 0; nt < NT; ++nt) accb[nt][q] = 0.f;
+        for (int mt = 0; mt < (GRAM ? MT : 1); ++mt) { accn[mt][0][q] = 0.f; accn[mt][1][q] = 0.f; }
+#pragma unroll
+        for (int nt = 0; nt < (GRAM ? NT : 1); ++nt) accb[nt][q] = 0.f;
     }
 
     // split K: warp w takes 64-byte blocks w, w + 8, ...; kMmaStages - 1 blocks are in flight per warp
@@ -300,9 +300,7 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
                                     (w + nb * kMmaWarps) * 4 + tig, units, lane);
         cp_async_commit();
         cp_async_wait<kMmaStages - 1>();         // block b has landed (each lane waits for its own copies)
-        MmaStage<MT, NT> sg;
-        mma_read_stage<MT, NT>(sg, wring + (b % kMmaStages) * PIECES * 32, lane);
-        mma_compute_stage<MT, NT>(sg, acc, accn, accb);
+        mma_consume_stage<MT, NT, GRAM>(wring + (b % kMmaStages) * PIECES * 32, lane, acc, accn, accb);
     }
     cp_async_wait<0>();
     __syncthreads();                             // every warp is done with its ring: reuse it for the partials
@@ -318,7 +316,7 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
             s_part[w][mt * 16 + g + 8][nt * 8 + 2 * tig + 1] = acc[mt][nt][3];
         }
     // Gram diagonals: the lane with tig == g / 2 holds entry (g, g) in c0 / c1 and (g + 8, g) in c2 / c3
-    if (tig == (g >> 1)) {
+    if (GRAM && tig == (g >> 1)) {
         const bool odd = g & 1;
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt) {
@@ -336,7 +334,7 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
         for (int ww = 0; ww < kMmaWarps; ++ww) d += (&s_part[ww][0][0])[idx];
         (&s_dot[0][0])[idx] = d;
     }
-    if (tid < FR + NC) {                                 // 1 / max(||x||, floor), warps added in warp order
+    if (GRAM && tid < FR + NC) {                         // 1 / max(||x||, floor), warps added in warp order
         float n2 = 0.f;
 #pragma unroll
         for (int ww = 0; ww < kMmaWarps; ++ww) n2 += tid < FR ? s_na[ww][tid] : s_nb[ww][tid - FR];
@@ -370,11 +368,39 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
     trace_mark(asrc.hdr, 2, true);
 }
 
+// r <= 1: 32 frames per CTA, norms from Gram diagonals, 96 registers (see TTF_MMA_BOUNDS)
+template <int MT, int NT>
+__global__ void TTF_MMA_BOUNDS
+k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t, AnchorSrc asrc,
+            float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt)
+{
+    match_mma_body<MT, NT, true, kMmaStagesDefault>(X, F, H, W, C, r, t, asrc, nullptr, 0, shat, dst, keep, cnt);
+}
+
+// r = 2: the 25 candidate rows of a cell are as much data as 25 source rows, so a CTA takes 64 frames per cell to
+// amortise them (2.6 -> 1.4 times |X| of operand traffic); norms come from the sweep, which frees the registers
+// of the Gram accumulators for the 64 x 32 tile of dot products.
+#ifndef TTF_WIDE_MT
+#define TTF_WIDE_MT 4
+#endif
+#ifndef TTF_WIDE_STAGES
+#define TTF_WIDE_STAGES 2
+#endif
+constexpr int kWideMT = TTF_WIDE_MT;
+constexpr int kWideStages = TTF_WIDE_STAGES;
+__global__ void __launch_bounds__(kMmaWarps * 32, 2)
+k_match_mma_wide(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t, AnchorSrc asrc,
+                 const float* __restrict__ ssq, int nslice,
+                 float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt)
+{
+    match_mma_body<kWideMT, 4, false, kWideStages>(X, F, H, W, C, r, t, asrc, ssq, nslice, shat, dst, keep, cnt);
+}
+
 template <int MT, int NT>
 static cudaError_t launch_mma_t(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                                 unsigned char* keep, cudaStream_t st) {
     const long long chunks = (p.F + 16 * MT - 1) / (16 * MT);
-    constexpr size_t smem = sizeof(uint4) * kMmaWarps * kMmaStages * (2 * MT + NT) * 32;
+    constexpr size_t smem = sizeof(uint4) * kMmaWarps * kMmaStagesDefault * (2 * MT + NT) * 32;
     static bool configured = false;              // per instantiation; the attribute belongs to the function
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(k_match_mma<MT, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -390,6 +416,28 @@ static cudaError_t launch_mma_t(const Problem& p, const Scratch& s, int* out_anc
     cfg.attrs = attr; cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, k_match_mma<MT, NT>, reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C,
                               p.r, p.t, make_anchor_src(p, s, out_anchor), shat, dst, keep, s.cnt);
+}
+
+static cudaError_t launch_mma_wide(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
+                                   unsigned char* keep, cudaStream_t st) {
+    constexpr size_t smem = sizeof(uint4) * kMmaWarps * kWideStages * (2 * kWideMT + 4) * 32;
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(k_match_mma_wide, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    const long long chunks = (p.F + 16 * kWideMT - 1) / (16 * kWideMT);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(chunks * p.N)); cfg.blockDim = dim3(kMmaWarps * 32);
+    cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, k_match_mma_wide, reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r,
+                              p.t, make_anchor_src(p, s, out_anchor), (const float*)s.ssq, p.nslice, shat, dst, keep,
+                              s.cnt);
 }
 
 template <typename T, int V>
@@ -416,7 +464,7 @@ cudaError_t launch_match(const Problem& p, const Scratch& s, int* out_anchor, fl
     if (uses_mma_match(p)) {
         if (p.r == 0) return launch_mma_t<2, 1>(p, s, out_anchor, shat, dst, keep, st);
         if (p.r == 1) return launch_mma_t<2, 2>(p, s, out_anchor, shat, dst, keep, st);
-        return launch_mma_t<1, 4>(p, s, out_anchor, shat, dst, keep, st);     // 25 candidates: 16 frames per CTA
+        return launch_mma_wide(p, s, out_anchor, shat, dst, keep, st);
     }
     return p.vec ? launch_generic_t<bf16_t, 8>(p, s, out_anchor, shat, dst, keep, st)
                  : launch_generic_t<bf16_t, 1>(p, s, out_anchor, shat, dst, keep, st);
