@@ -39,7 +39,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="vl8b_cal")
     ap.add_argument("--clips", type=int, default=16, help="distinct clips per step (batch)")
-    ap.add_argument("--streams", type=int, default=4, help="CUDA streams the clips of a step are spread over")
+    ap.add_argument("--streams", type=int, default=0,
+                    help="0: one ttf_compress_batch call per step (the library spreads the clips over its own four "
+                         "streams); S > 0: one ttf_compress call per clip on S streams of the caller")
     ap.add_argument("--threshold", type=float, default=None)
     ap.add_argument("--anchor", default="auto", choices=["auto", "first", "last"], help="anchor rule")
     ap.add_argument("--no-graph", action="store_true",
@@ -275,8 +277,13 @@ def main():
     joins = [torch.cuda.Event() for _ in streams]
 
     amode = {"auto": 0, "first": 1, "last": 2}[args.anchor]
+    if args.streams == 0 and amode != 0:
+        raise SystemExit("--anchor first/last needs --streams S > 0 (ttf_compress_batch uses the automatic anchor)")
 
     def step():
+        if args.streams == 0:
+            P.ttf_compress_batch(devX, spec.r, t, out_tok, out_cnt, out_pos, stream=main_stream)
+            return
         if nstreams == 1:
             for j in range(nclips):
                 P.ttf_compress(devX[j], spec.r, t, out_tok[j], out_cnt[j], out_pos[j], stream=main_stream,
@@ -339,34 +346,33 @@ def main():
     value = tokens_all / (ms_step * 1e-3)
     clips_per_s = value / FN
 
-    # ---- per-kernel durations: the same clips again, one stream, events around every launch, so that each
-    # kernel is timed alone (no other clip's kernels share the GPU with it) ----------------------------------
-    prof_steps = min(args.steps, 50)
-    P.ttf_profile_begin()
-    for _ in range(prof_steps):
-        for j in range(nclips):
-            P.ttf_compress(devX[j], spec.r, t, out_tok[j], out_cnt[j], out_pos[j], stream=main_stream,
-                           anchor_mode=amode)
-    torch.cuda.synchronize()
-    prof = P.ttf_profile_end()
+    # ---- per-kernel durations at steady state: every kernel launched back to back for all clips of the step,
+    # CUDA events (on the launching stream) around each group, divided by the clips; the batch is larger than L2,
+    # so every launch finds its clip cold in HBM, as it does with several clips in flight --------------------
     sampler.stop()
     clocks = sampler.summary(w0, w1)
-
-    launches_per_step = sum(v[1] for v in prof.values()) // prof_steps
-    kern = {k: {"launches": v[1], "us_per_launch": 1e3 * v[0] / v[1]} for k, v in prof.items() if v[1]}
-    tot = sum(v[0] for v in prof.values())
-    dominant = max(kern, key=lambda k: prof[k][0])
+    kernel_ms = P.ttf_profile_stages(devX, spec.r, t, out_tok, out_cnt, out_pos, reps=min(args.steps, 20),
+                                     stream=main_stream)
+    torch.cuda.synchronize()
+    launches_per_step = 4 * nclips if amode == 0 else 3 * nclips
+    kern = {k: {"us_per_launch": 1e3 * v} for k, v in kernel_ms.items() if v > 0}
+    tot = sum(kernel_ms.values())
+    dominant = max(kern, key=lambda k: kernel_ms[k])
     peak_gbs, peak_kind = peaks()
     avg_count = sum(counts) / nclips
     kbytes = A.kernel_bytes(dominant, spec.F, spec.N, C, spec.itemsize, int(round(avg_count)))
     achieved = kbytes / (kern[dominant]["us_per_launch"] * 1e-6) / 1e9
-    roofline = {"bound": "hbm", "kernel": dominant, "timed": "alone, single stream, CUDA events around each launch", "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
+    roofline = {"bound": "hbm", "kernel": dominant,
+                "timed": "each kernel launched back to back for the clips of a step (cold in HBM), CUDA events around the group, / clips",
+                "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
                 "frac": achieved / peak_gbs, "peak_source": f"of {peak_kind}",
                 "traffic": NCU_TRAFFIC.get((spec.name, dominant)) if amode == 0 else None,
-                "traffic_note": "ncu, cold caches (in the pipeline the second pass over X is served by L2 when one clip is in flight)",
+                "traffic_note": "ncu, cold caches, one launch",
                 "algorithmic_bytes_per_launch": kbytes,
-                "kernel_share": {k: prof[k][0] / tot for k in kern},
-                "kernel_us": {k: round(kern[k]["us_per_launch"], 3) for k in kern}}
+                "kernel_share": {k: kernel_ms[k] / tot for k in kern},
+                "kernel_us": {k: round(kern[k]["us_per_launch"], 3) for k in kern},
+                "kernel_frac": {k: A.kernel_bytes(k, spec.F, spec.N, C, spec.itemsize, int(round(avg_count)))
+                                / (kern[k]["us_per_launch"] * 1e-6) / 1e9 / peak_gbs for k in kern}}
     bmin = A.pass_bytes(spec.F, spec.N, C, spec.itemsize, int(round(avg_count)))
     pass_gbs = bmin * nclips / (ms_step * 1e-3) / 1e9
     pass_roofline = {"bytes_per_clip": bmin, "achieved": pass_gbs, "unit": "GB/s", "frac_of_measured_copy": pass_gbs / peak_gbs,
@@ -408,7 +414,8 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(spec, t, nclips, nstreams, tokens_step, args.anchor, use_graph),
+            "config": workload_config(spec, t, nclips, "4 (library: ttf_compress_batch)" if args.streams == 0 else nstreams,
+                                      tokens_step, args.anchor, use_graph),
             "clips_per_s": clips_per_s, "rho": rho, "count_mean": avg_count,
             "roofline": roofline, "pass_roofline": pass_roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches_per_step * args.steps), "gpu_launches_per_step": int(launches_per_step),

@@ -89,6 +89,33 @@ int ttf_workspace_bytes(int F, int H, int W, int C, int r, int dtype, size_t* by
 int ttf_compress(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
                  void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream);
 
+/*
+ * A batch of clips of one shape in one call (the long-video workload: the clips of a request processed
+ * concurrently; Sec. 3 treats every clip independently, so this is scheduling only and each clip's results are
+ * exactly those of ttf_compress).  features, out_tokens, out_count and out_pos_thw are HOST arrays of nclips
+ * DEVICE pointers, read before the call returns.  The clips are spread round-robin over four streams that the
+ * library keeps per device; these fork from `stream` and join it again through events, so the call is
+ * asynchronous, ordered on `stream` like any other, and can be captured in a CUDA graph.  The kernels of one clip
+ * leave much of the GPU idle while they ramp up and drain; with four clips in flight those gaps are filled.
+ * Scratch: one block per internal stream, from the cache.
+ * With the single-launch pass switched on (ttf_set_single_launch) qualifying batches instead run as one persistent
+ * cooperative launch per 32 clips in which two groups of CTAs work on consecutive clips half a clip apart.
+ */
+int ttf_compress_batch(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
+                       int dtype, void* const* out_tokens, int* const* out_count, int* const* out_pos_thw,
+                       ttf_stream_t stream);
+
+/*
+ * Execution variant (the paper has no counterpart).  on != 0: bf16 clips with r <= 1, 16-byte aligned rows and at
+ * most 256 frames run the whole pass as ONE persistent cooperative kernel whose phases are separated by
+ * grid-wide barriers (bounded waits; a wait that gives up reports out_count = -1) instead of four kernels.  Results
+ * are identical except that the frame sums of Eq. (auto_anchor) are added in a different fixed order.  Off by
+ * default (or TTF_SINGLE_LAUNCH=1 in the environment): measured on B200 the kernel sequence is faster for the
+ * clip shapes of the paper; the single launch is for callers for whom the number of launches matters.
+ * Process-wide; returns the previous setting.
+ */
+int ttf_set_single_launch(int on);
+
 /* Same, with caller-owned scratch: `workspace` must be 256-byte aligned device memory of at least
  * ttf_workspace_bytes(...) bytes that no other in-flight call uses.  Allocates nothing. */
 int ttf_compress_ws(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
@@ -203,12 +230,24 @@ int ttf_query_static(const void* features, int F, int H, int W, int C, int r, fl
  * device time in milliseconds and the number of launches; `kinds` is the length of both arrays
  * (TTF_KERNEL_KINDS covers all).  Kinds: 0 frame-sum (and norm) sweep, 1 frame statistics of the anchor rule,
  * 2 windowed match + gate (its prologue takes the anchor arg max), 3 compaction gather (with the frame-count
- * prefix of clips longer than 1024 frames), 4 fuse-count bookkeeping of ttf_query.  Profiling is process-wide
+ * prefix of clips longer than 1024 frames), 4 fuse-count bookkeeping of ttf_query, 5 the single-launch pass.  Profiling is process-wide
  * and meant for benchmarks; leave it off otherwise.
  */
-#define TTF_KERNEL_KINDS 5
+#define TTF_KERNEL_KINDS 6
 int ttf_profile_begin(void);
 int ttf_profile_end(double* total_ms, long long* launches, int kinds);
+
+/*
+ * Steady-state duration of each kernel of the pass (no counterpart in the paper).  For `reps` rounds, each of the
+ * four kernels (kinds 0..3 above) is launched back to back for all `nclips` clips of the batch, each clip on its
+ * own scratch block, with one pair of CUDA events around the group; ms_per_launch[kind] = group time / nclips,
+ * averaged over the rounds.  With a batch larger than L2 every launch finds its clip cold in HBM, which is how a
+ * kernel runs when several clips are in flight.  Arguments as ttf_compress_batch; the outputs are those of the
+ * pass.  Always the kernel sequence, whatever ttf_set_single_launch says.  Synchronises `stream`.
+ */
+int ttf_profile_stages(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
+                       int dtype, void* const* out_tokens, int* const* out_count, int* const* out_pos_thw,
+                       int reps, double* ms_per_launch, int kinds, ttf_stream_t stream);
 
 /* Frees every cached scratch / staging buffer of the calling process (all devices).  Synchronises. */
 int ttf_release(void);

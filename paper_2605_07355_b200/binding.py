@@ -22,11 +22,11 @@ EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
     "ttf_query_static", "ttf_compress_ex", "ttf_query_ex", "ttf_compress_segment", "ttf_restore",
-    "ttf_sim_histogram",
+    "ttf_sim_histogram", "ttf_compress_batch", "ttf_set_single_launch", "ttf_profile_stages",
 ]
 TTF_ANCHOR_AUTO, TTF_ANCHOR_FIRST, TTF_ANCHOR_LAST, TTF_ANCHOR_EXPLICIT = 0, 1, 2, 3
 TTF_STATIC_SCRATCH_BYTES = 8 << 20
-KERNEL_KINDS = ["norm_sum", "frame_stats", "match", "compact", "fuse_count"]
+KERNEL_KINDS = ["norm_sum", "frame_stats", "match", "compact", "fuse_count", "single_launch"]
 
 _lib = None
 
@@ -57,6 +57,12 @@ def lib() -> ctypes.CDLL:
         L.ttf_workspace_bytes.argtypes = shape + [i, ctypes.POINTER(sz)]
         L.ttf_compress.restype = i
         L.ttf_compress.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp]
+        L.ttf_compress_batch.restype = i
+        L.ttf_compress_batch.argtypes = [vp, i] + shape + [f, i, vp, vp, vp, vp]
+        L.ttf_profile_stages.restype = i
+        L.ttf_profile_stages.argtypes = [vp, i] + shape + [f, i, vp, vp, vp, i, ctypes.POINTER(ctypes.c_double), i, vp]
+        L.ttf_set_single_launch.restype = i
+        L.ttf_set_single_launch.argtypes = [i]
         L.ttf_compress_ws.restype = i
         L.ttf_compress_ws.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, sz, vp]
         L.ttf_query.restype = i
@@ -157,6 +163,58 @@ def ttf_compress(features: torch.Tensor, r: int, t: float, out_tokens: Optional[
                                        _p(workspace), workspace.numel() * workspace.element_size(), sp)
     if rc != TTF_OK:
         raise TTFError(rc, "ttf_compress")
+    return out_tokens, out_count, out_pos_thw
+
+
+def ttf_profile_stages(features, r: int, t: float, out_tokens, out_count, out_pos_thw, reps: int = 10, stream=None) -> dict:
+    """ttf_profile_stages: milliseconds per launch of each kernel of the pass at steady state, by kernel kind."""
+    feats = list(features)
+    F, H, W, C = _check_features(feats[0], "cuda")
+    B = len(feats)
+    arr = lambda ts: (ctypes.c_void_p * B)(*[t_.data_ptr() for t_ in ts])
+    n = len(KERNEL_KINDS)
+    ms = (ctypes.c_double * n)()
+    with torch.cuda.device(feats[0].device):
+        rc = lib().ttf_profile_stages(arr(feats), B, F, H, W, C, int(r), float(t), _dtype_code(feats[0]),
+                                      arr(out_tokens), arr(out_count), arr(out_pos_thw), int(reps), ms, n,
+                                      _stream_ptr(stream))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_profile_stages")
+    return {k: float(ms[i]) for i, k in enumerate(KERNEL_KINDS[:4])}
+
+
+def ttf_set_single_launch(on: bool) -> bool:
+    """ttf_set_single_launch: switches the one-kernel variant of the pass on or off; returns the previous setting."""
+    return bool(lib().ttf_set_single_launch(1 if on else 0))
+
+
+def ttf_compress_batch(features, r: int, t: float, out_tokens=None, out_count=None, out_pos_thw=None, stream=None):
+    """ttf_compress_batch: `features` is a sequence of [F, H, W, C] device tensors of one shape and dtype.
+    Returns three lists (out_tokens, out_count, out_pos_thw), one entry per clip, as ttf_compress does for one
+    clip.  Does not synchronise."""
+    feats = list(features)
+    if not feats:
+        raise ValueError("empty batch")
+    F, H, W, C = _check_features(feats[0], "cuda")
+    dev, dt = feats[0].device, feats[0].dtype
+    for x in feats[1:]:
+        if _check_features(x, "cuda") != (F, H, W, C) or x.dtype != dt or x.device != dev:
+            raise ValueError("all clips of a batch must have the same shape, dtype and device")
+    n, B = F * H * W, len(feats)
+    if out_tokens is None:
+        out_tokens = [torch.empty((n, C), dtype=dt, device=dev) for _ in range(B)]
+    if out_count is None:
+        out_count = [torch.empty(1, dtype=torch.int32, device=dev) for _ in range(B)]
+    if out_pos_thw is None:
+        out_pos_thw = [torch.empty((n, 3), dtype=torch.int32, device=dev) for _ in range(B)]
+    if not (len(out_tokens) == len(out_count) == len(out_pos_thw) == B):
+        raise ValueError("one output of each kind per clip")
+    arr = lambda ts: (ctypes.c_void_p * B)(*[t_.data_ptr() for t_ in ts])
+    with torch.cuda.device(dev):
+        rc = lib().ttf_compress_batch(arr(feats), B, F, H, W, C, int(r), float(t), _dtype_code(feats[0]),
+                                      arr(out_tokens), arr(out_count), arr(out_pos_thw), _stream_ptr(stream))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_compress_batch")
     return out_tokens, out_count, out_pos_thw
 
 

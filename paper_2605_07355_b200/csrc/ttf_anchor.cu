@@ -148,8 +148,10 @@ static cudaError_t launch_sum_t(const Problem& p, const Scratch& s, cudaStream_t
     const unsigned blocks = (unsigned)((long long)p.F * p.nq);
     const dim3 g(blocks), b(kNormThreads);
     if (!needs_sweep_norms(p))
-        return launch_pdl(k_norm_sum<T, V, 32, false>, g, b, st, X, p.F, p.N, p.C, p.nq, s.S, s.ssq, s.cnt, s.hdr);
-    return launch_pdl(k_norm_sum<T, V, 32, true>, g, b, st, X, p.F, p.N, p.C, p.nq, s.S, s.ssq, s.cnt, s.hdr);
+        return launch_ex(true, 0, k_norm_sum<T, V, 32, false>, g, b, st, X, p.F, p.N, p.C, p.nq, s.S,
+                         s.ssq, s.cnt, s.hdr);
+    return launch_ex(true, 0, k_norm_sum<T, V, 32, true>, g, b, st, X, p.F, p.N, p.C, p.nq, s.S, s.ssq,
+                     s.cnt, s.hdr);
 }
 
 // ---------------------------------------------------------------------------------------------------------

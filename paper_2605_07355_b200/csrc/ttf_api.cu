@@ -4,6 +4,7 @@
 #include "ttf_internal.cuh"
 
 #include <cmath>
+#include <cstdlib>
 #include <map>
 #include <mutex>
 #include <utility>
@@ -33,7 +34,7 @@ int sm_count() {
 }
 
 // ---- optional per-kernel timing: CUDA events recorded around every launch while profiling is on ---------
-enum { PK_NORM_SUM = 0, PK_FRAME_STATS = 1, PK_MATCH = 2, PK_COMPACT = 3, PK_FUSE_COUNT = 4, PK_KINDS = 5 };
+enum { PK_NORM_SUM = 0, PK_FRAME_STATS = 1, PK_MATCH = 2, PK_COMPACT = 3, PK_FUSE_COUNT = 4, PK_FUSED = 5, PK_KINDS = 6 };
 struct ProfRecord { int kind; cudaEvent_t a, b; };
 static std::mutex g_prof_mu;
 static bool g_prof_on = false;
@@ -64,7 +65,7 @@ void carve_scratch(const Problem& p, void* base, Scratch* s) {
     s->hdr = (int*)take(sizeof(int) * kHdrInts);      // control words first: one small memset clears them
     s->cnt = (int*)take(sizeof(int) * p.F);
     s->prefix = (int*)take(sizeof(int) * ((size_t)p.F + 1));
-    s->S = (float*)take(sizeof(float) * (size_t)p.F * p.C);
+    s->S = (float*)take(sizeof(float) * (size_t)p.F * p.C * (fused_eligible(p) ? kFusedMaxSplit : 1));
     s->Dp = (float*)take(sizeof(float) * (size_t)kStatReplicas * p.nsl * p.F);
     s->Qp = (float*)take(sizeof(float) * (size_t)kStatReplicas * p.nsl * p.F);
     s->Gp = (float*)take(sizeof(float) * (size_t)kStatReplicas * p.nsl);
@@ -162,10 +163,28 @@ static int run_front(const Problem& p, const Scratch& s, int* out_anchor, float*
     return TTF_OK;
 }
 
+// 1: clips that qualify take the single-launch pass (ttf_fused.cu); 0: the kernel sequence.  Off unless
+// TTF_SINGLE_LAUNCH=1 is in the environment or ttf_set_single_launch(1) was called: on the clips measured so far
+// the kernel sequence spread over streams is the faster of the two.
+static int g_use_fused = -1;
+static bool use_fused(const Problem& p, const void* out_tokens) {
+    if (g_use_fused < 0) {
+        const char* e = getenv("TTF_SINGLE_LAUNCH");
+        g_use_fused = (e && e[0] == '1') ? 1 : 0;
+    }
+    return g_use_fused == 1 && fused_eligible(p) && reinterpret_cast<uintptr_t>(out_tokens) % 16 == 0;
+}
+
 static int compress_impl(const Problem& p, void* ws, void* out_tokens, int* out_count, int* out_pos,
                          cudaStream_t st) {
     Scratch s;
     carve_scratch(p, ws, &s);
+    if (use_fused(p, out_tokens)) {
+        cudaError_t e;
+        { ProfScope ps(st, PK_FUSED);
+          e = launch_fused(p, s, nullptr, s.shat, s.dst, s.keep, s.fuse_cnt, out_tokens, out_pos, out_count, st); }
+        return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+    }
     int rc = run_front(p, s, nullptr, s.shat, s.dst, s.keep, st);
     if (rc != TTF_OK) return rc;
     cudaError_t e;
@@ -181,6 +200,12 @@ static int query_impl(const Problem& p, void* ws, int* out_anchor, unsigned char
     float* shat = out_sim ? out_sim : s.shat;
     int* dst = out_dst ? out_dst : s.dst;
     unsigned char* keep = out_keep ? out_keep : s.keep;
+    if (use_fused(p, nullptr)) {
+        cudaError_t e;
+        { ProfScope ps(st, PK_FUSED);
+          e = launch_fused(p, s, out_anchor, shat, dst, keep, out_fuse, nullptr, nullptr, nullptr, st); }
+        return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+    }
     int rc = run_front(p, s, out_anchor, shat, dst, keep, st);
     if (rc != TTF_OK) return rc;
     if (out_fuse) {
@@ -374,6 +399,94 @@ int ttf_query_ex(const void* features, int F, int H, int W, int C, int r, float 
     return query_impl(p, ws, out_anchor, out_keep, out_dst, out_best_sim, out_fuse_cnt, (cudaStream_t)stream);
 }
 
+// ---- batches on the library's own streams -----------------------------------------------------------------
+// The clips of a batch are independent, and the kernels of one clip leave most of the GPU idle while they ramp up
+// and drain, so a batch is spread round-robin over kBatchStreams internal streams per device that fork from the
+// caller's stream and join it again (events only: the call stays asynchronous and can be captured in a graph).
+constexpr int kBatchStreams = 4;
+struct BatchLanes { cudaStream_t s[kBatchStreams] = {}; cudaEvent_t fork = nullptr; cudaEvent_t join[kBatchStreams] = {}; bool ok = false; };
+static std::map<int, BatchLanes> g_lanes;
+
+static int batch_lanes(BatchLanes** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    std::lock_guard<std::mutex> lk(g_mu);
+    BatchLanes& L = g_lanes[dev];
+    if (!L.ok) {
+        e = cudaEventCreateWithFlags(&L.fork, cudaEventDisableTiming);
+        for (int i = 0; i < kBatchStreams && e == cudaSuccess; ++i) {
+            e = cudaStreamCreateWithFlags(&L.s[i], cudaStreamNonBlocking);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&L.join[i], cudaEventDisableTiming);
+        }
+        if (e != cudaSuccess) return cuda_fail(e);
+        L.ok = true;
+    }
+    *out = &L;
+    return TTF_OK;
+}
+
+static int batch_on_streams(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
+                            int dtype, void* const* out_tokens, int* const* out_count, int* const* out_pos_thw,
+                            cudaStream_t st) {
+    BatchLanes* L = nullptr;
+    int rc = batch_lanes(&L);
+    if (rc != TTF_OK) return rc;
+    const int lanes = nclips < kBatchStreams ? nclips : kBatchStreams;
+    cudaError_t e = cudaEventRecord(L->fork, st);
+    for (int i = 0; i < lanes && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(L->s[i], L->fork, 0);
+    if (e != cudaSuccess) return cuda_fail(e);
+    int first_rc = TTF_OK;
+    for (int n = 0; n < nclips && first_rc == TTF_OK; ++n)
+        first_rc = ttf_compress(features[n], F, H, W, C, r, t, dtype, out_tokens[n], out_count[n], out_pos_thw[n],
+                                (ttf_stream_t)L->s[n % lanes]);
+    // always join, also after a failed launch, so that the caller's stream (or capture) is whole again
+    for (int i = 0; i < lanes; ++i) {
+        cudaError_t e2 = cudaEventRecord(L->join[i], L->s[i]);
+        if (e2 == cudaSuccess) e2 = cudaStreamWaitEvent(st, L->join[i], 0);
+        if (e2 != cudaSuccess && e == cudaSuccess) e = e2;
+    }
+    if (first_rc != TTF_OK) return first_rc;
+    return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+}
+
+int ttf_set_single_launch(int on) {
+    const int before = g_use_fused == 1 ? 1 : 0;
+    g_use_fused = on ? 1 : 0;
+    return before;
+}
+
+int ttf_compress_batch(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
+                       int dtype, void* const* out_tokens, int* const* out_count, int* const* out_pos_thw,
+                       ttf_stream_t stream) {
+    if (!features || !out_tokens || !out_count || !out_pos_thw || nclips < 1) return TTF_ERR_INVALID_ARG;
+    for (int n = 0; n < nclips; ++n)
+        if (!features[n] || !out_tokens[n] || !out_count[n] || !out_pos_thw[n]) return TTF_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    Problem p;
+    int rc = make_problem(features[0], F, H, W, C, r, t, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    bool batched = nclips > 1 && use_fused(p, out_tokens[0]) && !g_prof_on;
+    for (int n = 1; n < nclips && batched; ++n)
+        batched = reinterpret_cast<uintptr_t>(features[n]) % 16 == 0 && reinterpret_cast<uintptr_t>(out_tokens[n]) % 16 == 0;
+    Scratch s;
+    carve_scratch(p, nullptr, &s);
+    const size_t stride = s.bytes;
+    const int chunk = nclips < kFusedBatchMax ? nclips : kFusedBatchMax;
+    if (!batched) return batch_on_streams(features, nclips, F, H, W, C, r, t, dtype, out_tokens, out_count, out_pos_thw, st);
+    void* ws = nullptr;
+    rc = cached_scratch(stride * chunk, st, &ws);
+    if (rc != TTF_OK) return rc;
+    carve_scratch(p, ws, &s);
+    for (int base = 0; base < nclips; base += kFusedBatchMax) {
+        const int m = nclips - base < kFusedBatchMax ? nclips - base : kFusedBatchMax;
+        cudaError_t e = launch_fused_batch(p, s, (long long)stride, m, features + base, out_tokens + base,
+                                           out_pos_thw + base, out_count + base, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return TTF_OK;
+}
+
 int ttf_compress_segment(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
                          int frame_base, void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream) {
     if (!features || !out_tokens || !out_count || !out_pos_thw) return TTF_ERR_INVALID_ARG;
@@ -502,6 +615,58 @@ int ttf_profile_end(double* total_ms, long long* launches, int kinds) {
     return first == cudaSuccess ? TTF_OK : cuda_fail(first);
 }
 
+int ttf_profile_stages(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
+                       int dtype, void* const* out_tokens, int* const* out_count, int* const* out_pos_thw,
+                       int reps, double* ms_per_launch, int kinds, ttf_stream_t stream) {
+    if (!features || !out_tokens || !out_count || !out_pos_thw || !ms_per_launch || nclips < 1 || reps < 1 ||
+        kinds < 4) return TTF_ERR_INVALID_ARG;
+    for (int n = 0; n < nclips; ++n)
+        if (!features[n] || !out_tokens[n] || !out_count[n] || !out_pos_thw[n]) return TTF_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    std::vector<Problem> ps(nclips);
+    for (int n = 0; n < nclips; ++n) {
+        int rc = make_problem(features[n], F, H, W, C, r, t, dtype, &ps[n]);
+        if (rc != TTF_OK) return rc;
+    }
+    Scratch s0;
+    carve_scratch(ps[0], nullptr, &s0);
+    size_t stride = s0.bytes;
+    for (int n = 1; n < nclips; ++n) {           // (the layout depends on the alignment of the clip)
+        Scratch sn;
+        carve_scratch(ps[n], nullptr, &sn);
+        if (sn.bytes > stride) stride = sn.bytes;
+    }
+    void* ws = nullptr;
+    int rc = cached_scratch(stride * nclips, st, &ws);
+    if (rc != TTF_OK) return rc;
+    cudaEvent_t ev[5];
+    for (auto& e : ev) if (cudaEventCreate(&e) != cudaSuccess) return cuda_fail(cudaGetLastError());
+    for (int k = 0; k < kinds; ++k) ms_per_launch[k] = 0.0;
+    cudaError_t e = cudaSuccess;
+    for (int rep = 0; rep < reps && e == cudaSuccess; ++rep) {
+        for (int stage = 0; stage < 4 && e == cudaSuccess; ++stage) {
+            cudaEventRecord(ev[stage], st);
+            for (int n = 0; n < nclips && e == cudaSuccess; ++n) {
+                Scratch s;
+                carve_scratch(ps[n], (char*)ws + stride * n, &s);
+                if (stage == 0) e = launch_norm_sum(ps[n], s, st);
+                else if (stage == 1) e = launch_frame_stats(ps[n], s, nullptr, st);
+                else if (stage == 2) e = launch_match(ps[n], s, nullptr, s.shat, s.dst, s.keep, st);
+                else e = launch_compact(ps[n], s, out_tokens[n], out_pos_thw[n], out_count[n], st);
+            }
+        }
+        cudaEventRecord(ev[4], st);
+        if (e == cudaSuccess) e = cudaEventSynchronize(ev[4]);
+        for (int stage = 0; stage < 4 && e == cudaSuccess; ++stage) {
+            float ms = 0.f;
+            e = cudaEventElapsedTime(&ms, ev[stage], ev[stage + 1]);
+            ms_per_launch[stage] += ms / (double)nclips / (double)reps;
+        }
+    }
+    for (auto& x : ev) cudaEventDestroy(x);
+    return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+}
+
 int ttf_release(void) {
     std::lock_guard<std::mutex> lk(g_mu);
     int cur = 0;
@@ -526,6 +691,16 @@ int ttf_release(void) {
         if (s.stream) cudaStreamDestroy(s.stream);
     }
     g_staging.clear();
+    for (auto& kv : g_lanes) {
+        cudaSetDevice(kv.first);
+        BatchLanes& L = kv.second;
+        for (int i = 0; i < kBatchStreams; ++i) {
+            if (L.s[i]) { cudaStreamSynchronize(L.s[i]); cudaStreamDestroy(L.s[i]); }
+            if (L.join[i]) cudaEventDestroy(L.join[i]);
+        }
+        if (L.fork) cudaEventDestroy(L.fork);
+    }
+    g_lanes.clear();
     cudaSetDevice(cur);
     return first == cudaSuccess ? TTF_OK : cuda_fail(first);
 }

@@ -10,10 +10,9 @@
 // the survivors are spread over the frames.  No warp ever waits for another one.
 #include "ttf_internal.cuh"
 #include "ttf_async.cuh"
+#include "ttf_gather.cuh"
 
 namespace ttf {
-
-constexpr int kCopyWarps = 8;
 
 // exclusive scan of the effective per-frame counts (anchor frame counts as 0) for clips with more frames
 // than fit the shared-memory scan of the gather kernel
@@ -66,115 +65,6 @@ template <> struct CopyUnit<2> { using type = uint16_t; };
 #define TTF_COPY_UNROLL 8
 #endif
 constexpr int kCopyUnroll = TTF_COPY_UNROLL;   // 16-byte units in flight per lane (two steps for an 8 KB row)
-constexpr int kScanChunks = 4;       // frame counts per lane fetched at once by the warp-level frame search
-
-// Tokens fused into each anchor cell j: |{(k,i): k != a, keep = 0, dst = j}|, gather-side (every cell looks at
-// the (2r+1)^2 x (F-1) tokens that can point to it), integer, fixed order.  Run by whole CTAs: block `b` of `nb`.
-__device__ __forceinline__ void fuse_count_cta(int F, int H, int W, int r, int a, const unsigned char* keep,
-                                               const int* dst, int* fuse_cnt, int b, int nb) {
-    if (fuse_cnt == nullptr) return;
-    const int N = H * W;
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    for (int j = b * kCopyWarps + w; j < N; j += nb * kCopyWarps) {
-        const int y = j / W, x = j - y * W;
-        int c = 0;
-        for (int k = lane; k < F; k += 32) {
-            if (k == a) continue;
-            for (int yy = max(0, y - r); yy <= min(H - 1, y + r); ++yy)
-                for (int xx = max(0, x - r); xx <= min(W - 1, x + r); ++xx) {
-                    const size_t f = (size_t)k * N + yy * W + xx;
-                    c += (!__ldcg(keep + f) && __ldcg(dst + f) == j) ? 1 : 0;
-                }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-        if (lane == 0) fuse_cnt[j] = c;
-    }
-}
-
-// Frame search of the gather: the frame that holds the e-th preserved source token (flat order, anchor frame
-// skipped) and the number of preserved tokens before that frame.  Returns the total P; k_out = -1 when e is past
-// the end (e < 0 asks for the total only).  All lanes of a warp call it with the same arguments.
-__device__ __forceinline__ int find_frame(const int* __restrict__ cnt, const int* __restrict__ gprefix, int F, int a,
-                                          int lane, int e, int& k_out, int& before) {
-    int running = 0;
-    k_out = -1; before = 0;
-    if (F > kWarpPrefixMaxF) {                         // pre-scanned prefix: binary search
-        int lo = 0, hi = F;
-        const int P = __ldcg(gprefix + F);
-        if (e < P) {
-            while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (__ldcg(gprefix + mid) <= e) lo = mid; else hi = mid; }
-            k_out = lo; before = __ldcg(gprefix + lo);
-        }
-        return P;
-    }
-    for (int base = 0; base < F; base += 32 * kScanChunks) {
-        int c[kScanChunks];
-#pragma unroll
-        for (int q = 0; q < kScanChunks; ++q) {
-            const int k = base + q * 32 + lane;
-            c[q] = (k < F && k != a) ? __ldcg(cnt + k) : 0;
-        }
-#pragma unroll
-        for (int q = 0; q < kScanChunks; ++q) {
-            int incl = c[q];
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int v = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += v;
-            }
-            const int total = __shfl_sync(0xffffffffu, incl, 31);
-            if (k_out < 0 && e < running + total) {
-                const unsigned m = __ballot_sync(0xffffffffu, running + incl > e);
-                const int l = __ffs(m) - 1;
-                k_out = base + q * 32 + l;
-                before = running + __shfl_sync(0xffffffffu, incl - c[q], l);
-            }
-            running += total;
-        }
-        if (k_out >= 0 && e >= 0) break;               // e < 0 asks for the total only
-    }
-    return running;
-}
-
-
-// Cell index of the n-th (0-based) retained token of one frame: a warp-wide rank/select over the keep flags.
-// All lanes must call with the same arguments; returns -1 if the frame holds fewer than n+1 retained tokens.
-__device__ __forceinline__ int select_in_frame(const unsigned char* __restrict__ kf, int N, int n, int lane) {
-    for (int b = 0; b < N; b += 256) {                     // 8 cells per lane, 256 per step
-        const int c0 = b + lane * 8;
-        unsigned bits = 0;
-        if (c0 + 8 <= N && ((reinterpret_cast<uintptr_t>(kf + c0) & 7) == 0)) {
-            const uint2 v = __ldcg(reinterpret_cast<const uint2*>(kf + c0));
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                bits |= ((v.x >> (8 * e)) & 0xffu) ? (1u << e) : 0u;
-                bits |= ((v.y >> (8 * e)) & 0xffu) ? (1u << (4 + e)) : 0u;
-            }
-        } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) bits |= (c0 + e < N && __ldcg(kf + c0 + e) != 0) ? (1u << e) : 0u;
-        }
-        const int mine = __popc(bits);
-        int incl = mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        const int total = __shfl_sync(0xffffffffu, incl, 31);
-        if (n < total) {
-            const int excl = incl - mine;
-            const bool here = n >= excl && n < incl;       // exactly one lane
-            const int cell = here ? c0 + (int)__fns(bits, 0, n - excl + 1) : 0;
-            const unsigned who = __ballot_sync(0xffffffffu, here);
-            return __shfl_sync(0xffffffffu, cell, __ffs(who) - 1);
-        }
-        n -= total;
-    }
-    return -1;
-}
-
 // Gather with bulk asynchronous copies, for rows that are 16-byte aligned multiples of 16 bytes: a warp finds the
 // source row of its output row as above, then one lane moves the row global -> shared -> global with two bulk
 // copies per piece of at most kBulkPiece bytes, so no data passes through registers.
@@ -356,15 +246,9 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
             if (e != cudaSuccess) return e;
             configured = true;
         }
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = g; cfg.blockDim = b; cfg.dynamicSmemBytes = smem; cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
-        return cudaLaunchKernelEx(&cfg, k_compact_bulk, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,
-                                  (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep,
-                                  (const int*)s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy, NA, p.pos_t_offset);
+        return launch_ex(pdl, smem, k_compact_bulk, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r,
+                         (const int*)s.hdr, (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep,
+                         (const int*)s.dst, out, out_pos, out_count, s.fuse_cnt, ncopy, NA, p.pos_t_offset);
     }
     if (esize == 4)
         return launch_pdl_if(pdl, k_compact<4>, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,

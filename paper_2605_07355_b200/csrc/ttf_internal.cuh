@@ -13,10 +13,13 @@ constexpr int kWarpPrefixMaxF = 1024;  // frame counts up to this are scanned by
 constexpr int kHdrInts = 64;
 constexpr int kStatReplicas = 16;      // copies of the frame statistics, so that the CTAs that read them at the
                                        // same moment do not all queue on the same few cache lines
+constexpr int kFusedMaxSplit = 4;     // fused pass: at most this many token ranges per frame in the sweep
 constexpr int kResolveMaxF = 256;      // clips up to this many frames: the matching kernel takes the arg max itself
 
 // header words of the scratch block
-enum { HDR_ANCHOR = 0, HDR_DONE_ALL = 1, HDR_ERROR = 2 };   // HDR_ERROR: a bounded wait gave up
+enum { HDR_ANCHOR = 0, HDR_DONE_ALL = 1, HDR_ERROR = 2,     // HDR_ERROR: a bounded wait gave up
+       HDR_BAR = 3, HDR_SWEEP = 5, HDR_EXIT = 6 };           // fused pass: barrier arrivals of the (two) CTA groups, CTAs
+                                                             // that completed a sweep, CTAs done; zero between calls
 
 // Problem description handed to every launcher.
 struct Problem {
@@ -42,7 +45,7 @@ struct Scratch {
     int* hdr;           // [kHdrInts]  anchor frame, arrival counter of the anchor-pick slices
     int* cnt;           // [F]   preserved tokens per source frame (Eq. gating summed over a frame)
     int* prefix;        // [F+1] exclusive scan of cnt, only used when F > kWarpPrefixMaxF
-    float* S;           // [F, C] per-frame channel sums
+    float* S;           // [F, C] per-frame channel sums ([kFusedMaxSplit, F, C] token-range parts in the fused pass)
     float* Dp;          // [kStatReplicas][nsl, F] per-slice share of <S_k, g>
     float* Qp;          // [kStatReplicas][nsl, F] per-slice share of |S_k|^2
     float* Gp;          // [kStatReplicas][nsl]    per-slice share of |g|^2
@@ -96,6 +99,19 @@ cudaError_t launch_restore(const void* comp, size_t row_bytes, int F, int N, con
 cudaError_t launch_sim_histogram(const float* sim, const int* anchor, int F, int N, int bins, unsigned int* hist,
                                  cudaStream_t st);
 
+// The whole pass in one cooperative launch (ttf_fused.cu).  out_tokens == NULL stops before the compaction.
+bool fused_eligible(const Problem& p);
+int fused_grid();                       // CTAs of the fused kernel on the current device
+void set_fused_ctas_per_sm(int n);      // 1 or 2
+cudaError_t launch_fused(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
+                         unsigned char* keep, int* fuse_cnt, void* out_tokens, int* out_pos, int* out_count,
+                         cudaStream_t st);
+
+constexpr int kFusedBatchMax = 32;      // clips per launch of the batched pass
+cudaError_t launch_fused_batch(const Problem& p, const Scratch& s, long long ws_stride, int nclips,
+                               const void* const* X, void* const* out_tokens, int* const* out_pos,
+                               int* const* out_count, cudaStream_t st);
+
 int sm_count();   // SMs of the current device (cached per device)
 
 inline AnchorSrc make_anchor_src(const Problem& p, const Scratch& s, int* out_anchor) {
@@ -113,15 +129,24 @@ inline AnchorSrc make_anchor_src(const Problem& p, const Scratch& s, int* out_an
 // produces is NOT read-only data for it: it must be read with L2-coherent loads (__ldcg), never through the
 // non-coherent / L1 path that `const __restrict__` pointers and __ldg select.  Only X is truly read-only.
 template <typename... KArgs, typename... Args>
+inline cudaError_t launch_ex(bool pdl, size_t smem, void (*kernel)(KArgs...), dim3 grid, dim3 block,
+                             cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    int n = 0;
+    if (pdl) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr; cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl_if(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st,
                                  Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    return launch_ex(pdl, 0, kernel, grid, block, st, args...);
 }
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, cudaStream_t st, Args... args) {

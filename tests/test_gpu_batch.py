@@ -1,0 +1,104 @@
+"""GPU parity of the batch entry point and of the single-launch variant of the pass (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ttf_oracle as O
+from paper_2605_07355_b200 import clips
+import paper_2605_07355_b200 as P
+from tests.parity import check_clip, to_device, to_bits
+from tests.test_gpu_parity import corr_clip
+
+pytestmark = pytest.mark.gpu
+
+
+def assert_same_as_single(Xs, r, t, outs):
+    """every clip of a batch must give exactly what ttf_compress gives for it alone"""
+    toks, cnts, poss = outs
+    for j, X in enumerate(Xs):
+        a = P.ttf_compress(X, r, t)
+        torch.cuda.synchronize()
+        L = int(a[1].item())
+        assert int(cnts[j].item()) == L, (j, int(cnts[j].item()), L)
+        assert torch.equal(toks[j][:L], a[0][:L]) and torch.equal(poss[j][:L], a[2][:L]), j
+
+
+@pytest.fixture
+def single_launch():
+    before = P.ttf_set_single_launch(True)
+    yield
+    P.ttf_set_single_launch(before)
+
+
+def test_batch_on_library_streams_matches_single_calls_and_oracle():
+    s = clips.CONFIGS["vl2b_cal"]
+    Xn = [clips.make_clip(s, s.seed + j) for j in range(7)]          # 7 clips over 4 streams: ragged last round
+    Xs = [to_device(x) for x in Xn]
+    outs = P.ttf_compress_batch(Xs, s.r, s.t)
+    torch.cuda.synchronize()
+    assert_same_as_single(Xs, s.r, s.t, outs)
+    R = O.compress(Xn[3], s.r, s.t)
+    q = P.ttf_query(Xs[3], s.r, s.t)
+    forced = O.compress(Xn[3], s.r, s.t, anchor_frame=int(q["anchor"].item()), forced_keep=q["keep"].cpu().numpy())
+    in_band = np.abs(R.s_hat.astype(np.float32) - np.float32(s.t)) < 1e-4
+    assert not ((q["keep"].cpu().numpy() != R.keep) & ~in_band).any()
+    L = int(outs[1][3].item())
+    assert L == forced.count
+    assert (outs[2][3][:L].cpu().numpy() == forced.pos).all() and (to_bits(outs[0][3][:L]) == forced.tokens).all()
+
+
+def test_batch_small_and_fp32_and_stream_order():
+    Xs = [to_device(corr_clip(3, 4, 5, 40, seed=31 + j, dtype="f32")) for j in range(3)]
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        outs = P.ttf_compress_batch(Xs, 1, 0.7, stream=st)
+        first = outs[1][0] + 0                   # ordered after the batch on the caller's stream
+    st.synchronize()
+    assert_same_as_single(Xs, 1, 0.7, outs)
+    assert int(first.item()) == int(outs[1][0].item())
+    one = P.ttf_compress_batch(Xs[:1], 1, 0.7)
+    torch.cuda.synchronize()
+    assert_same_as_single(Xs[:1], 1, 0.7, one)
+    with pytest.raises(ValueError):
+        P.ttf_compress_batch([Xs[0], Xs[1][:2]], 1, 0.7)
+
+
+SHAPES = [(1, 4, 4, 32, 1), (2, 3, 5, 40, 1), (6, 5, 6, 264, 0), (17, 3, 3, 72, 1), (33, 2, 3, 8, 1),
+          (9, 4, 6, 1032, 1), (40, 7, 9, 512, 1)]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+def test_single_launch_small_shapes(single_launch, shape):
+    F, H, W, C, r = shape
+    X = corr_clip(F, H, W, C, seed=sum(shape), dtype="bf16")
+    for t in (0.7, 0.5):
+        check_clip(X, r, t)
+
+
+def test_single_launch_paper_shaped_and_fixed_anchors(single_launch):
+    s = clips.CONFIGS["vl2b_cal"]
+    rep = check_clip(clips.make_clip(s), s.r, s.t)
+    assert abs(rep["rho"] - 0.67) < 0.02
+    X = corr_clip(5, 6, 7, 256, seed=5, dtype="bf16")
+    for mode, frame in ((1, 0), (2, 0), (3, 2)):
+        rep = check_clip(X, 1, 0.7, anchor_mode=mode, anchor_frame=frame)
+        assert rep["anchor"] == {1: 0, 2: 4, 3: 2}[mode]
+    check_clip(np.zeros((3, 3, 3, 16), np.uint16), 1, 0.5)           # all-zero bf16 clip
+
+
+def test_single_launch_batch_two_groups():
+    s = clips.CONFIGS["vl2b_cal"]
+    Xs = [to_device(clips.make_clip(s, s.seed + j)) for j in range(5)]      # odd count: the groups end unevenly
+    ref = [P.ttf_compress(x, s.r, s.t) for x in Xs]
+    torch.cuda.synchronize()
+    before = P.ttf_set_single_launch(True)
+    try:
+        for rep in range(2):                     # twice: the control words must be back at zero after a launch
+            toks, cnts, poss = P.ttf_compress_batch(Xs, s.r, s.t)
+            torch.cuda.synchronize()
+            for j in range(len(Xs)):
+                L = int(ref[j][1].item())
+                assert int(cnts[j].item()) == L
+                assert torch.equal(toks[j][:L], ref[j][0][:L]) and torch.equal(poss[j][:L], ref[j][2][:L])
+    finally:
+        P.ttf_set_single_launch(before)
