@@ -26,6 +26,8 @@
  * grid equals an all-pairs search done with scipy's cdist; a planted integer shift gives dst in closed form;
  * a frame equal to the clip mean wins the anchor rule with cosine 1; clip-and-mask equals window-intersect-
  * grid; rho is monotone in t and in r; survivors keep their (k, y, x) in ascending order.
+ * Mean fusion (ttf_oracle_fuse_mean, not the paper's method) is pinned by: nothing fused or identical frames give
+ * the anchor rows back; the weighted means add up to the sum of all absorbed tokens; numpy's own accumulation.
  * Parity unpinned: nothing computed here; what cannot be pinned is accuracy on real video, which needs the
  * paper's datasets and weights and is not computed by this file at all.
  */
@@ -262,4 +264,35 @@ void ttf_oracle_sim_histogram(const float* s_hat, int F, int N, int a, int bins,
 }
 
 /* Cache-aware Decode Alignment, Eqs. (Lpre), (decode_pos): pos_dec(l) = L' + T + l */
+/*
+ * Mean fusion.  NOT the paper's method: Sec. 3 (Threshold Gating) states that a fused token is replaced by its
+ * anchor token unchanged, with no convex combination of features.  This is the averaging alternative the paper
+ * contrasts itself with, written out as its plain definition so that the optional mean-fuse mode of the CUDA
+ * library has something to be checked against: anchor cell j receives the arithmetic mean of its own token and
+ * of every source token fused into it,
+ *     out_j = ( x_{a,j} + sum_{(k,i): keep(k,i) = 0, dst(k,i) = j} x_{k,i} ) / ( 1 + fuse_cnt_j ),
+ * in double.  out is [N, C].
+ */
+void ttf_oracle_fuse_mean(const float* X, int F, int N, int C, int a, const uint8_t* keep, const int* dst,
+                          double* out) {
+    int* members = (int*)malloc(sizeof(int) * (size_t)N);
+    for (int j = 0; j < N; ++j) {
+        members[j] = 1;
+        for (int c = 0; c < C; ++c) out[(size_t)j * C + c] = (double)X[((size_t)a * N + j) * C + c];
+    }
+    for (int k = 0; k < F; ++k) {
+        if (k == a) continue;
+        for (int i = 0; i < N; ++i) {
+            const size_t f = (size_t)k * N + i;
+            if (keep[f]) continue;
+            const int j = dst[f];
+            members[j] += 1;
+            for (int c = 0; c < C; ++c) out[(size_t)j * C + c] += (double)X[f * C + c];
+        }
+    }
+    for (int j = 0; j < N; ++j)
+        for (int c = 0; c < C; ++c) out[(size_t)j * C + c] /= (double)members[j];
+    free(members);
+}
+
 long long ttf_oracle_decode_pos(long long L_prime, long long T, long long l) { return L_prime + T + l; }

@@ -51,6 +51,8 @@ def _load():
         lib.ttf_oracle_restore.argtypes = [vp, c_sz, vp, vp, c_int, c_int, c_int, vp, vp]
         lib.ttf_oracle_sim_histogram.restype = None
         lib.ttf_oracle_sim_histogram.argtypes = [vp, c_int, c_int, c_int, c_int, vp]
+        lib.ttf_oracle_fuse_mean.restype = None
+        lib.ttf_oracle_fuse_mean.argtypes = [vp, c_int, c_int, c_int, c_int, vp, vp, vp]
         lib.ttf_oracle_decode_pos.restype = ctypes.c_longlong
         lib.ttf_oracle_decode_pos.argtypes = [ctypes.c_longlong] * 3
         _lib = lib
@@ -172,6 +174,33 @@ def compress_segment(X: np.ndarray, r: int, t: float, frame_base: int, forced_ke
     pos = R.pos[N:].copy()
     pos[:, 0] += frame_base - 1
     return R.tokens[N:], pos, R.count - N
+
+
+def fuse_mean(X: np.ndarray, keep: np.ndarray, dst: np.ndarray, a: int) -> np.ndarray:
+    """Mean fusion (NOT the paper's method, which replaces a fused token by its anchor token unchanged): [N, C]
+    f64, row j = mean of anchor token j and of the source tokens fused into it."""
+    F, H, W, C = _shape(X)
+    Xf = _widen(X)
+    keep = np.ascontiguousarray(keep, dtype=np.uint8)
+    dst = np.ascontiguousarray(dst, dtype=np.int32)
+    out = np.empty((H * W, C), dtype=np.float64)
+    _load().ttf_oracle_fuse_mean(_ptr(Xf), F, H * W, C, int(a), _ptr(keep), _ptr(dst), _ptr(out))
+    return out
+
+
+def round_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    """float64 -> bf16 bit patterns (uint16), round to nearest, ties to even, in one rounding."""
+    x = np.asarray(x, dtype=np.float64)
+    down = (x.astype(np.float32).view(np.uint32) & np.uint32(0xFFFF0000))          # a bf16 value near x
+    cand = np.stack([down - np.uint32(0x10000), down, down + np.uint32(0x10000)])     # its neighbours
+    vals = cand.view(np.float32).astype(np.float64)
+    err = np.abs(vals - x[None])
+    err = np.where(np.isfinite(vals), err, np.inf)
+    even = ((cand >> np.uint32(16)) & np.uint32(1)) == 0
+    nearest = err == err.min(axis=0)[None]
+    best = np.argmin(np.where(nearest, np.where(even, 0, 1), 2), axis=0)             # ties: the even pattern
+    out = np.take_along_axis(cand, best[None], axis=0)[0]
+    return (out >> np.uint32(16)).astype(np.uint16)
 
 
 def decode_pos(L_prime: int, T: int, l: int) -> int:

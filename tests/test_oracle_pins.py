@@ -322,3 +322,56 @@ def test_segment_emits_only_new_preserved_tokens():
     t_all, p_all, P_all = O.compress_segment(X, 1, 1.5, frame_base=0)    # nothing fused: all new frames, in order
     assert P_all == (F - 1) * N and (t_all == X[1:].reshape(-1, C)).all()
     assert O.compress_segment(np.repeat(X[:1], 3, axis=0), 1, 0.7, 5)[2] == 0
+
+
+# ---- mean fusion (the averaging alternative that Sec. 3, Threshold Gating, rules out; optional mode only) --------
+def test_mean_fuse_hand_example():
+    # F = 2 frames, N = 2 cells, C = 1; frame 0 is the anchor.  Both source tokens are fused into cell 0.
+    X = np.array([[[[1.0], [10.0]]], [[[3.0], [5.0]]]], np.float32)           # [F=2, H=1, W=2, C=1]
+    keep = np.array([1, 1, 0, 0], np.uint8)
+    dst = np.array([0, 1, 0, 0], np.int32)
+    out = O.fuse_mean(X, keep, dst, 0)
+    assert out.tolist() == [[3.0], [10.0]]                                    # (1 + 3 + 5) / 3 and 10 / 1
+    keep[3] = 1                                                               # a retained token contributes nothing
+    assert O.fuse_mean(X, keep, dst, 0).tolist() == [[2.0], [10.0]]
+    dst[2] = 1                                                                # ... and dst picks the receiving cell
+    assert O.fuse_mean(X, keep, dst, 0).tolist() == [[1.0], [6.5]]
+
+
+def test_mean_fuse_without_fusion_and_with_identical_frames_is_the_anchor_frame():
+    X = corr_clip(4, 5, 4, 24, seed=41)
+    R = O.compress(X, 1, 2.0)                                                 # t > 1: nothing is fused
+    assert (O.fuse_mean(X, R.keep, R.dst, R.anchor) == X[R.anchor].reshape(20, 24).astype(np.float64)).all()
+    Y = np.repeat(X[:1], 5, axis=0)                                           # identical frames: every mean is the row
+    R = O.compress(Y, 1, 0.7)
+    assert R.count == 20
+    assert (O.fuse_mean(Y, R.keep, R.dst, R.anchor) == Y[0].reshape(20, 24).astype(np.float64)).all()
+
+
+@pytest.mark.parametrize("seed,r", [(51, 0), (52, 1), (53, 2)])
+def test_mean_fuse_conserves_the_absorbed_mass_and_matches_numpy(seed, r):
+    F, H, W, C = 6, 5, 6, 40
+    N = H * W
+    X = corr_clip(F, H, W, C, seed=seed)
+    R = O.compress(X, r, 0.6)
+    assert 0 < (R.keep == 0).sum() < (F - 1) * N
+    out = O.fuse_mean(X, R.keep, R.dst, R.anchor)
+    flat = X.reshape(F * N, C).astype(np.float64)
+    fused = R.keep == 0
+    # the size-weighted means add up to everything that was absorbed: the anchor frame plus the fused tokens
+    total = (out * (1 + R.fuse_cnt)[:, None]).sum(axis=0)
+    assert np.allclose(total, flat[R.anchor * N:(R.anchor + 1) * N].sum(axis=0) + flat[fused].sum(axis=0), rtol=0, atol=1e-9)
+    # numpy's own scatter-add over the same (keep, dst)
+    acc = flat[R.anchor * N:(R.anchor + 1) * N].copy()
+    np.add.at(acc, R.dst[fused], flat[fused])
+    assert np.allclose(out, acc / (1 + np.bincount(R.dst[fused], minlength=N))[:, None], rtol=0, atol=1e-12)
+
+
+def test_bf16_rounding_helper_is_round_to_nearest_even():
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal(50000).astype(np.float32)
+    u = x.view(np.uint32)
+    rne = ((u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) >> np.uint32(16)).astype(np.uint16)
+    assert (O.round_to_bf16_bits(x.astype(np.float64)) == rne).all()
+    ties = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -1.0 - 3 * 2.0 ** -8])
+    assert O.round_to_bf16_bits(ties).tolist() == [0x3F80, 0x3F82, 0xBF82]
