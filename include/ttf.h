@@ -155,6 +155,19 @@ int ttf_query_ex(const void* features, int F, int H, int W, int C, int r, float 
                  int* out_fuse_cnt, ttf_stream_t stream);
 
 /*
+ * ttf_compress with MEAN fusion.  This is NOT the paper's method: Sec. 3 (Threshold Gating) replaces a fused token
+ * by its anchor token unchanged and states that there is no convex combination of features.  This entry point is
+ * the averaging alternative for callers who want to compare the two: everything is as in ttf_compress (same
+ * anchor, matches, gate, order, positions, L'), except that anchor row j of out_tokens holds
+ *     ( x_{a,j} + sum of the source tokens (k,i) with keep(k,i) = 0 and dst(k,i) = j ) / ( 1 + fuse_cnt_j ),
+ * accumulated in fp32 in ascending flat order k*N + i starting from the anchor token, divided once, and rounded to
+ * the clip's dtype (bf16: round to nearest even).  The reduction is segmented by anchor cell and uses no atomics,
+ * so results are reproducible bit for bit.  Preserved source rows are bit copies as before.
+ */
+int ttf_compress_mean(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                      void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream);
+
+/*
  * Streaming segment (Discussion D3: the last frame of each segment serves as a rolling anchor; new frames are
  * compressed against it and appended to the KV cache).  features = [F, H, W, C] whose frame 0 is the rolling
  * anchor, i.e. the last frame of the previous segment, which the consumer already holds; frames 1..F-1 are the

@@ -22,7 +22,7 @@ EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
     "ttf_query_static", "ttf_compress_ex", "ttf_query_ex", "ttf_compress_segment", "ttf_restore",
-    "ttf_sim_histogram", "ttf_compress_batch", "ttf_set_single_launch", "ttf_profile_stages",
+    "ttf_sim_histogram", "ttf_compress_batch", "ttf_set_single_launch", "ttf_profile_stages", "ttf_compress_mean",
 ]
 TTF_ANCHOR_AUTO, TTF_ANCHOR_FIRST, TTF_ANCHOR_LAST, TTF_ANCHOR_EXPLICIT = 0, 1, 2, 3
 TTF_STATIC_SCRATCH_BYTES = 8 << 20
@@ -63,6 +63,8 @@ def lib() -> ctypes.CDLL:
         L.ttf_profile_stages.argtypes = [vp, i] + shape + [f, i, vp, vp, vp, i, ctypes.POINTER(ctypes.c_double), i, vp]
         L.ttf_set_single_launch.restype = i
         L.ttf_set_single_launch.argtypes = [i]
+        L.ttf_compress_mean.restype = i
+        L.ttf_compress_mean.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp]
         L.ttf_compress_ws.restype = i
         L.ttf_compress_ws.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, sz, vp]
         L.ttf_query.restype = i
@@ -186,6 +188,23 @@ def ttf_profile_stages(features, r: int, t: float, out_tokens, out_count, out_po
 def ttf_set_single_launch(on: bool) -> bool:
     """ttf_set_single_launch: switches the one-kernel variant of the pass on or off; returns the previous setting."""
     return bool(lib().ttf_set_single_launch(1 if on else 0))
+
+
+def ttf_compress_mean(features: torch.Tensor, r: int, t: float, stream=None):
+    """ttf_compress_mean: ttf_compress with the anchor rows replaced by the means of the tokens fused into them
+    (not the paper's method).  Returns (out_tokens, out_count, out_pos_thw).  Does not synchronise."""
+    F, H, W, C = _check_features(features, "cuda")
+    dev = features.device
+    n = F * H * W
+    out_tokens = torch.empty((n, C), dtype=features.dtype, device=dev)
+    out_count = torch.empty(1, dtype=torch.int32, device=dev)
+    out_pos_thw = torch.empty((n, 3), dtype=torch.int32, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ttf_compress_mean(_p(features), F, H, W, C, int(r), float(t), _dtype_code(features),
+                                     _p(out_tokens), _p(out_count), _p(out_pos_thw), _stream_ptr(stream))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_compress_mean")
+    return out_tokens, out_count, out_pos_thw
 
 
 def ttf_compress_batch(features, r: int, t: float, out_tokens=None, out_count=None, out_pos_thw=None, stream=None):

@@ -399,6 +399,24 @@ int ttf_query_ex(const void* features, int F, int H, int W, int C, int r, float 
     return query_impl(p, ws, out_anchor, out_keep, out_dst, out_best_sim, out_fuse_cnt, (cudaStream_t)stream);
 }
 
+int ttf_compress_mean(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
+                      void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream) {
+    if (!features || !out_tokens || !out_count || !out_pos_thw) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    Scratch s;
+    carve_scratch(p, nullptr, &s);
+    void* ws = nullptr;
+    rc = cached_scratch(s.bytes, (cudaStream_t)stream, &ws);
+    if (rc != TTF_OK) return rc;
+    rc = compress_impl(p, ws, out_tokens, out_count, out_pos_thw, (cudaStream_t)stream);
+    if (rc != TTF_OK) return rc;
+    carve_scratch(p, ws, &s);
+    cudaError_t e = launch_fuse_mean(p, s, out_tokens, (cudaStream_t)stream);
+    return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+}
+
 // ---- batches on the library's own streams -----------------------------------------------------------------
 // The clips of a batch are independent, and the kernels of one clip leave most of the GPU idle while they ramp up
 // and drain, so a batch is spread round-robin over kBatchStreams internal streams per device that fork from the

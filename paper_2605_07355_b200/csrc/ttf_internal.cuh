@@ -99,6 +99,9 @@ cudaError_t launch_restore(const void* comp, size_t row_bytes, int F, int N, con
 cudaError_t launch_sim_histogram(const float* sim, const int* anchor, int F, int N, int bins, unsigned int* hist,
                                  cudaStream_t st);
 
+// Optional mean fusion (ttf_fuse.cu; not the paper's method): overwrites the anchor block of out_tokens.
+cudaError_t launch_fuse_mean(const Problem& p, const Scratch& s, void* out_tokens, cudaStream_t st);
+
 // The whole pass in one cooperative launch (ttf_fused.cu).  out_tokens == NULL stops before the compaction.
 bool fused_eligible(const Problem& p);
 int fused_grid();                       // CTAs of the fused kernel on the current device
