@@ -208,6 +208,17 @@ int ttf_compress_host(const void* features_host, int F, int H, int W, int C, int
                       void* out_tokens_host, int* out_count_host, int* out_pos_thw_host);
 
 /*
+ * ttf_compress_host for a batch of clips of one shape: features_host, out_tokens_host and out_pos_thw_host are
+ * arrays of nclips HOST pointers (pinned memory makes the copies asynchronous and lets them overlap), and
+ * out_count_host is an array of nclips ints that receives each clip's L'.  The clips go through two sets of
+ * device staging buffers: while clip n runs and its results are copied back, clip n + 1 is already being copied
+ * in, so the link to the host is busy in both directions.  Returns after everything has arrived.
+ */
+int ttf_compress_host_batch(const void* const* features_host, int nclips, int F, int H, int W, int C, int r, float t,
+                            int dtype, void* const* out_tokens_host, int* out_count_host,
+                            int* const* out_pos_thw_host);
+
+/*
  * ttf_query for callers that must not allocate device memory.  (The paper has no counterpart: this entry
  * point exists for the needs of the host program, not of the method.)
  *

@@ -22,7 +22,7 @@ EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
     "ttf_query_static", "ttf_compress_ex", "ttf_query_ex", "ttf_compress_segment", "ttf_restore",
-    "ttf_sim_histogram", "ttf_compress_batch", "ttf_set_single_launch", "ttf_profile_stages", "ttf_compress_mean",
+    "ttf_sim_histogram", "ttf_compress_batch", "ttf_set_single_launch", "ttf_profile_stages", "ttf_compress_mean", "ttf_compress_host_batch",
 ]
 TTF_ANCHOR_AUTO, TTF_ANCHOR_FIRST, TTF_ANCHOR_LAST, TTF_ANCHOR_EXPLICIT = 0, 1, 2, 3
 TTF_STATIC_SCRATCH_BYTES = 8 << 20
@@ -65,6 +65,8 @@ def lib() -> ctypes.CDLL:
         L.ttf_set_single_launch.argtypes = [i]
         L.ttf_compress_mean.restype = i
         L.ttf_compress_mean.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp]
+        L.ttf_compress_host_batch.restype = i
+        L.ttf_compress_host_batch.argtypes = [vp, i] + shape + [f, i, vp, vp, vp]
         L.ttf_compress_ws.restype = i
         L.ttf_compress_ws.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, sz, vp]
         L.ttf_query.restype = i
@@ -348,6 +350,35 @@ def ttf_compress_host(features: torch.Tensor, r: int, t: float, out_tokens: Opti
         raise TTFError(rc, "ttf_compress_host")
     L = int(cnt.value)
     return out_tokens[:L], L, out_pos_thw[:L]
+
+
+def ttf_compress_host_batch(features, r: int, t: float, out_tokens=None, out_pos_thw=None, device: Optional[int] = None):
+    """ttf_compress_host_batch: a sequence of HOST clips of one shape (pinned memory recommended) through the
+    pipelined copy-in / pass / copy-out path.  Returns (list of out_tokens[:L'], list of L', list of
+    out_pos_thw[:L']); synchronous."""
+    feats = list(features)
+    if not feats:
+        raise ValueError("empty batch")
+    F, H, W, C = _check_features(feats[0], "cpu")
+    for x in feats[1:]:
+        if _check_features(x, "cpu") != (F, H, W, C) or x.dtype != feats[0].dtype:
+            raise ValueError("all clips of a batch must have the same shape and dtype")
+    n, B = F * H * W, len(feats)
+    if out_tokens is None:
+        out_tokens = [torch.empty((n, C), dtype=feats[0].dtype) for _ in range(B)]
+    if out_pos_thw is None:
+        out_pos_thw = [torch.empty((n, 3), dtype=torch.int32) for _ in range(B)]
+    if len(out_tokens) != B or len(out_pos_thw) != B:
+        raise ValueError("one output of each kind per clip")
+    arr = lambda ts: (ctypes.c_void_p * B)(*[t_.data_ptr() for t_ in ts])
+    counts = (ctypes.c_int * B)()
+    with torch.cuda.device(torch.cuda.current_device() if device is None else device):
+        rc = lib().ttf_compress_host_batch(arr(feats), B, F, H, W, C, int(r), float(t), _dtype_code(feats[0]),
+                                           arr(out_tokens), ctypes.cast(counts, ctypes.c_void_p), arr(out_pos_thw))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_compress_host_batch")
+    Ls = [int(c) for c in counts]
+    return [o[:L] for o, L in zip(out_tokens, Ls)], Ls, [o[:L] for o, L in zip(out_pos_thw, Ls)]
 
 
 def ttf_release() -> None:

@@ -607,6 +607,111 @@ int ttf_compress_host(const void* features_host, int F, int H, int W, int C, int
     return TTF_OK;
 }
 
+// ---- host-buffer batch: copies in, kernels and copies out of consecutive clips overlap ----------------------
+struct HostPipe {
+    struct Slot { void* feat = nullptr; void* tok = nullptr; int* pos = nullptr; int* count = nullptr;
+                  cudaEvent_t loaded = nullptr, computed = nullptr, drained = nullptr; } slot[2];
+    size_t row_cap = 0, rows_cap = 0;            // capacity of the slot buffers: bytes per row, rows
+    cudaStream_t up = nullptr, run = nullptr, down = nullptr;
+    int* count_host = nullptr;                   // pinned, one int per slot
+    bool ok = false;
+};
+static std::map<int, HostPipe> g_pipes;
+static std::mutex g_pipe_mu;                     // one host batch at a time per process
+
+static cudaError_t pipe_prepare(HostPipe& hp, size_t FN, size_t row_bytes) {
+    cudaError_t e = cudaSuccess;
+    if (!hp.ok) {
+        e = cudaStreamCreateWithFlags(&hp.up, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&hp.run, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&hp.down, cudaStreamNonBlocking);
+        if (e == cudaSuccess) e = cudaHostAlloc((void**)&hp.count_host, 2 * sizeof(int), cudaHostAllocDefault);
+        for (auto& sl : hp.slot) {
+            if (e == cudaSuccess) e = cudaMalloc((void**)&sl.count, 256);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sl.loaded, cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sl.computed, cudaEventDisableTiming);
+            if (e == cudaSuccess) e = cudaEventCreateWithFlags(&sl.drained, cudaEventDisableTiming);
+        }
+        if (e != cudaSuccess) return e;
+        hp.ok = true;
+    }
+    if (hp.rows_cap * hp.row_cap < FN * row_bytes || hp.rows_cap < FN) {
+        e = cudaDeviceSynchronize();
+        for (auto& sl : hp.slot) {
+            if (sl.feat) cudaFree(sl.feat);
+            if (sl.tok) cudaFree(sl.tok);
+            if (sl.pos) cudaFree(sl.pos);
+            sl.feat = sl.tok = nullptr; sl.pos = nullptr;
+            if (e == cudaSuccess) e = cudaMalloc(&sl.feat, FN * row_bytes);
+            if (e == cudaSuccess) e = cudaMalloc(&sl.tok, FN * row_bytes);
+            if (e == cudaSuccess) e = cudaMalloc((void**)&sl.pos, FN * 3 * sizeof(int));
+        }
+        if (e != cudaSuccess) { hp.rows_cap = hp.row_cap = 0; return e; }
+        hp.rows_cap = FN; hp.row_cap = row_bytes;
+    }
+    return cudaSuccess;
+}
+
+int ttf_compress_host_batch(const void* const* features_host, int nclips, int F, int H, int W, int C, int r, float t,
+                            int dtype, void* const* out_tokens_host, int* out_count_host,
+                            int* const* out_pos_thw_host) {
+    if (!features_host || !out_tokens_host || !out_count_host || !out_pos_thw_host || nclips < 1) return TTF_ERR_INVALID_ARG;
+    for (int n = 0; n < nclips; ++n)
+        if (!features_host[n] || !out_tokens_host[n] || !out_pos_thw_host[n]) return TTF_ERR_INVALID_ARG;
+    Problem p;
+    int rc = make_problem(reinterpret_cast<const void*>(uintptr_t(256)), F, H, W, C, r, t, dtype, &p);
+    if (rc != TTF_OK) return rc;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    const size_t esize = dtype == TTF_DTYPE_F32 ? 4 : 2;
+    const size_t FN = (size_t)p.F * p.N, row_bytes = (size_t)C * esize;
+
+    std::lock_guard<std::mutex> lk(g_pipe_mu);
+    HostPipe& hp = g_pipes[dev];
+    e = pipe_prepare(hp, FN, row_bytes);
+    if (e != cudaSuccess) return cuda_fail(e);
+
+    auto load_and_run = [&](int n) -> int {      // copy clip n in and run the pass on it, all asynchronous
+        HostPipe::Slot& sl = hp.slot[n & 1];
+        cudaError_t e2 = cudaSuccess;
+        if (n >= 2) e2 = cudaStreamWaitEvent(hp.up, sl.drained, 0);          // the slot's last results have left
+        if (e2 == cudaSuccess) e2 = cudaMemcpyAsync(sl.feat, features_host[n], FN * row_bytes, cudaMemcpyHostToDevice, hp.up);
+        if (e2 == cudaSuccess) e2 = cudaEventRecord(sl.loaded, hp.up);
+        if (e2 == cudaSuccess) e2 = cudaStreamWaitEvent(hp.run, sl.loaded, 0);
+        if (e2 != cudaSuccess) return cuda_fail(e2);
+        int rc2 = ttf_compress(sl.feat, F, H, W, C, r, t, dtype, sl.tok, sl.count, sl.pos, (ttf_stream_t)hp.run);
+        if (rc2 != TTF_OK) return rc2;
+        e2 = cudaEventRecord(sl.computed, hp.run);
+        return e2 == cudaSuccess ? TTF_OK : cuda_fail(e2);
+    };
+
+    rc = load_and_run(0);
+    for (int n = 0; n < nclips && rc == TTF_OK; ++n) {
+        if (n + 1 < nclips) rc = load_and_run(n + 1);                        // next clip travels while this one drains
+        if (rc != TTF_OK) break;
+        HostPipe::Slot& sl = hp.slot[n & 1];
+        e = cudaStreamWaitEvent(hp.down, sl.computed, 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(hp.count_host + (n & 1), sl.count, sizeof(int), cudaMemcpyDeviceToHost, hp.down);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(hp.down);            // L' sizes the copies back
+        if (e != cudaSuccess) { rc = cuda_fail(e); break; }
+        const int Lp = hp.count_host[n & 1];
+        out_count_host[n] = Lp;
+        if (Lp < 0 || (size_t)Lp > FN) { rc = TTF_ERR_CUDA; break; }
+        e = cudaMemcpyAsync(out_tokens_host[n], sl.tok, (size_t)Lp * row_bytes, cudaMemcpyDeviceToHost, hp.down);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(out_pos_thw_host[n], sl.pos, (size_t)Lp * 3 * sizeof(int), cudaMemcpyDeviceToHost, hp.down);
+        if (e == cudaSuccess) e = cudaEventRecord(sl.drained, hp.down);
+        if (e != cudaSuccess) { rc = cuda_fail(e); break; }
+    }
+    // nothing of this call stays in flight, whatever happened
+    cudaError_t e1 = cudaStreamSynchronize(hp.up), e2 = cudaStreamSynchronize(hp.run), e3 = cudaStreamSynchronize(hp.down);
+    if (rc != TTF_OK) return rc;
+    if (e1 != cudaSuccess) return cuda_fail(e1);
+    if (e2 != cudaSuccess) return cuda_fail(e2);
+    if (e3 != cudaSuccess) return cuda_fail(e3);
+    return TTF_OK;
+}
+
 int ttf_profile_begin(void) {
     std::lock_guard<std::mutex> lk(g_prof_mu);
     for (auto& r : g_prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
@@ -709,6 +814,25 @@ int ttf_release(void) {
         if (s.stream) cudaStreamDestroy(s.stream);
     }
     g_staging.clear();
+    for (auto& kv : g_pipes) {
+        cudaSetDevice(kv.first);
+        HostPipe& hp = kv.second;
+        cudaDeviceSynchronize();
+        for (auto& sl : hp.slot) {
+            if (sl.feat) cudaFree(sl.feat);
+            if (sl.tok) cudaFree(sl.tok);
+            if (sl.pos) cudaFree(sl.pos);
+            if (sl.count) cudaFree(sl.count);
+            if (sl.loaded) cudaEventDestroy(sl.loaded);
+            if (sl.computed) cudaEventDestroy(sl.computed);
+            if (sl.drained) cudaEventDestroy(sl.drained);
+        }
+        if (hp.count_host) cudaFreeHost(hp.count_host);
+        if (hp.up) cudaStreamDestroy(hp.up);
+        if (hp.run) cudaStreamDestroy(hp.run);
+        if (hp.down) cudaStreamDestroy(hp.down);
+    }
+    g_pipes.clear();
     for (auto& kv : g_lanes) {
         cudaSetDevice(kv.first);
         BatchLanes& L = kv.second;

@@ -102,3 +102,44 @@ def test_single_launch_batch_two_groups():
                 assert torch.equal(toks[j][:L], ref[j][0][:L]) and torch.equal(poss[j][:L], ref[j][2][:L])
     finally:
         P.ttf_set_single_launch(before)
+
+
+def test_host_batch_matches_device_calls():
+    s = clips.CONFIGS["tiny_cal"]
+    Xn = [clips.make_clip(s, s.seed + j) for j in range(5)]           # more clips than staging slots
+    host = [torch.from_numpy(x).pin_memory() for x in Xn]
+    toks, Ls, poss = P.ttf_compress_host_batch(host, s.r, s.t)
+    for j, x in enumerate(Xn):
+        a = P.ttf_compress(to_device(x), s.r, s.t)
+        torch.cuda.synchronize()
+        L = int(a[1].item())
+        assert Ls[j] == L and torch.equal(toks[j], a[0][:L].cpu()) and torch.equal(poss[j], a[2][:L].cpu())
+    one_t, one_L, one_p = P.ttf_compress_host(host[2], s.r, s.t)
+    assert one_L == Ls[2] and torch.equal(one_t, toks[2]) and torch.equal(one_p, poss[2])
+
+
+def test_bench_configuration_full_size_against_oracle():
+    """the launch configuration the benchmark times: 16 clips of the 8B shape through one ttf_compress_batch call,
+    every clip checked against the oracle (decisions outside the threshold band exact, the rest bit for bit)"""
+    s = clips.CONFIGS["vl8b_cal"]
+    n = 16
+    Xn = [clips.make_clip(s, s.seed + j) for j in range(n)]
+    Xs = [to_device(x) for x in Xn]
+    for rep in range(2):                                               # second round: scratch reuse across calls
+        toks, cnts, poss = P.ttf_compress_batch(Xs, s.r, s.t)
+    torch.cuda.synchronize()
+    rhos = []
+    for j in range(n):
+        R = O.compress(Xn[j], s.r, s.t)
+        q = P.ttf_query(Xs[j], s.r, s.t)
+        keep = q["keep"].cpu().numpy()
+        assert int(q["anchor"].item()) == R.anchor
+        in_band = np.abs(R.s_hat.astype(np.float32) - np.float32(s.t)) < 1e-4
+        assert not ((keep != R.keep) & ~in_band).any()
+        forced = O.compress(Xn[j], s.r, s.t, anchor_frame=R.anchor, forced_keep=keep)
+        L = int(cnts[j].item())
+        assert L == forced.count
+        assert (poss[j][:L].cpu().numpy() == forced.pos).all()
+        assert (to_bits(toks[j][:L]) == forced.tokens).all()
+        rhos.append(1.0 - L / s.tokens)
+    assert abs(float(np.mean(rhos)) - 0.67) < 0.03
