@@ -6,8 +6,9 @@ the dominant kernel, end-to-end rate through the host-buffer entry point, and th
                     [--workload NAME] [--clips B] [--streams S] [--no-e2e] [--no-cpu]
 
 A step is one pass of the whole path (norm/frame-sum sweep, anchor pick, windowed match + gate, compaction
-with positions and fuse bookkeeping) over a batch of B distinct synthetic clips of the workload, one
-ttf_compress call per clip.  The batch is larger than L2, so every clip starts cold in HBM.  Rank 0 prints
+with positions and fuse bookkeeping) over a batch of B distinct synthetic clips of the workload: one
+ttf_compress_batch call (or, with --streams S, one ttf_compress call per clip on S streams of the caller).
+The batch is larger than L2, so every clip starts cold in HBM.  Rank 0 prints
 one JSON line.  With N > 1 (torchrun) every rank runs the same batch shape on its own GPU: clips are
 independent, there is no collective on the data path (weak scaling, replicas).
 """

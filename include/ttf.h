@@ -232,7 +232,7 @@ int ttf_compress_host_batch(const void* const* features_host, int nclips, int F,
  * so every GPU on which the library is used holds those 8 MiB until the process exits, whether or not this
  * function is ever called.  Arguments, outputs and results are exactly those of ttf_query.
  *   - A clip whose scratch need (the unaligned-layout figure ttf_workspace_bytes reports is an upper bound;
- *     the 8B-shaped clip F=32, 16x16, C=4096 bf16 needs about 1.3 MiB) exceeds the array is rejected with
+ *     the 8B-shaped clip F=32, 16x16, C=4096 bf16 needs about 3 MiB) exceeds the array is rejected with
  *     TTF_ERR_STATIC_LIMIT before anything is launched.
  *   - The first call on each device looks up the array's device address (a CUDA runtime query, no
  *     allocation); make that first call outside any stream capture.  Later calls only enqueue work:
