@@ -422,7 +422,7 @@ k_ttf_fused(const __grid_constant__ BatchArgs B)
             const int units = A.N * chunks;
             for (int u = rank; u < units; u += size) {
                 const int i = u % A.N, k0 = (u / A.N) * 32;
-                match_mma_unit<2, NT, true, kMmaStagesDefault>(A.X, A.F, A.H, A.W, A.C, A.r, A.t, a, i, k0, nullptr, 0,
+                match_mma_unit<2, NT, true, kMmaStagesDefault>(A.X, A.F, A.H, A.W, A.C, A.r, A.t, [a]() { return a; }, i, k0, nullptr, 0,
                                                               A.shat, A.dst, A.keep, A.cnt, dyn_smem);
                 __syncthreads();
             }

@@ -101,15 +101,21 @@ __device__ __forceinline__ void match_mma_body(const bf16_t* __restrict__ X, int
     const int k0 = (blockIdx.x / N) * 16 * MT;
     pdl_launch_dependents();
     trace_mark(asrc.hdr, 2, false);
-    pdl_wait();                                  // the frame statistics are complete (X itself is an input)
+    // Everything upstream is complete after this wait: the frame statistics, and also whatever produced X (an
+    // earlier kernel of the caller may still be writing X while this CTA is already resident, so X is not read
+    // before the wait either).
+    pdl_wait();
     trace_mark(asrc.hdr, 5, false);
-    const int a = resolve_anchor(asrc, F);
-    if (blockIdx.x == 0 && threadIdx.x == 0 && !asrc.from_hdr) {
-        asrc.hdr[HDR_ANCHOR] = a;                // the gather reads it from here
-        if (asrc.out_anchor) *asrc.out_anchor = a;
-    }
-    trace_mark(asrc.hdr, 4, true);
-    match_mma_unit<MT, NT, GRAM, ST>(X, F, H, W, C, r, t, a, i, k0, ssq, nslice, shat, dst, keep, cnt, dyn_smem);
+    auto anchor_fn = [&]() -> int {              // runs while the first source rows are in flight
+        const int a = resolve_anchor(asrc, F);
+        if (blockIdx.x == 0 && threadIdx.x == 0 && !asrc.from_hdr) {
+            asrc.hdr[HDR_ANCHOR] = a;            // the gather reads it from here
+            if (asrc.out_anchor) *asrc.out_anchor = a;
+        }
+        trace_mark(asrc.hdr, 4, true);
+        return a;
+    };
+    match_mma_unit<MT, NT, GRAM, ST>(X, F, H, W, C, r, t, anchor_fn, i, k0, ssq, nslice, shat, dst, keep, cnt, dyn_smem);
     trace_mark(asrc.hdr, 2, true);
 }
 

@@ -52,19 +52,24 @@ __device__ __forceinline__ void cp_async16(void* dst_smem, const void* src, bool
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// slot layout of a stage: [(2 MT + NT) pieces][32 lanes] x 16 bytes
-template <int MT, int NT>
+// slot layout of a stage: [(2 MT + NT) pieces][32 lanes] x 16 bytes.  DO_A / DO_B: copy the pieces of the source
+// rows / of the candidate rows (the prologue copies them at different times, see match_mma_unit)
+template <int MT, int NT, bool DO_A = true, bool DO_B = true>
 __device__ __forceinline__ void mma_issue_stage(uint4* slot, const uint4* const (&arow)[MT][2],
                                                 const uint4* const (&brow)[NT], const bool (&bvalid)[NT],
                                                 int idx, int units, int lane) {
     const bool ok = idx < units;
     const int safe = ok ? idx : 0;
+    if constexpr (DO_A) {
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt)
+        for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int h = 0; h < 2; ++h) cp_async16(slot + (mt * 2 + h) * 32 + lane, arow[mt][h] + safe, ok);
+            for (int h = 0; h < 2; ++h) cp_async16(slot + (mt * 2 + h) * 32 + lane, arow[mt][h] + safe, ok);
+    }
+    if constexpr (DO_B) {
 #pragma unroll
-    for (int nt = 0; nt < NT; ++nt) cp_async16(slot + (2 * MT + nt) * 32 + lane, brow[nt] + safe, ok && bvalid[nt]);
+        for (int nt = 0; nt < NT; ++nt) cp_async16(slot + (2 * MT + nt) * 32 + lane, brow[nt] + safe, ok && bvalid[nt]);
+    }
 }
 
 // Consumes one landed stage of a warp: dot products of every source row with every candidate row and, when
@@ -109,12 +114,15 @@ __device__ __forceinline__ void mma_consume_stage(const uint4* slot, int lane, f
 #define TTF_MMA_BOUNDS __maxnreg__(TTF_MMA_MAXREG)
 // GRAM: token norms from Gram-diagonal MMAs (else from the sweep's partial squared norms); ST: cp.async stages.
 //
-// One unit of work: cell i, frames k0 .. k0 + 16 MT - 1, anchor frame a.  Called by all threads of a CTA of
-// kMmaWarps warps; `dyn_smem` is at least kMmaWarps * ST * (2 MT + NT) * 512 bytes, 128-byte aligned.  A CTA that
-// runs several units in a row must put a __syncthreads() between them.
-template <int MT, int NT, bool GRAM, int ST>
+// One unit of work: cell i, frames k0 .. k0 + 16 MT - 1.  Called by all threads of a CTA of kMmaWarps warps;
+// `dyn_smem` is at least kMmaWarps * ST * (2 MT + NT) * 512 bytes, 128-byte aligned.  A CTA that runs several
+// units in a row must put a __syncthreads() between them.
+// The anchor frame comes from `anchor_fn()`, which every thread calls once, AFTER the copies of the source rows
+// of the first ST - 1 stages have been issued: the source rows do not depend on the anchor, so the loads that the
+// anchor arg max waits for overlap their flight.  X must be readable when the unit is entered.
+template <int MT, int NT, bool GRAM, int ST, typename AnchorFn>
 __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t,
-                                               int a, int i, int k0, const float* ssq, int nslice,
+                                               AnchorFn anchor_fn, int i, int k0, const float* ssq, int nslice,
                                                float* __restrict__ shat, int* __restrict__ dst,
                                                unsigned char* __restrict__ keep, int* __restrict__ cnt,
                                                unsigned char* dyn_smem)
@@ -149,15 +157,6 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
         return (yy >= 0 && yy < H && xx >= 0 && xx < W) ? yy * W + xx : -1;
     };
 
-    if (tid < NC) s_j[tid] = cand_index(tid);
-    if constexpr (!GRAM) {                       // inverse norms from the sweep's partials
-        const size_t FN = (size_t)F * N;
-        for (int q = tid; q < FR + NC; q += kMmaWarps * 32) {
-            if (q < FR) { const int k = k0 + q; s_rs[q] = k < F ? inv_norm(ssq, nslice, FN, (size_t)k * N + i) : 0.f; }
-            else { const int j = cand_index(q - FR); s_ra[q - FR] = j >= 0 ? inv_norm(ssq, nslice, FN, (size_t)a * N + j) : 0.f; }
-        }
-    }
-
     const uint4* arow[MT][2];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
@@ -166,8 +165,33 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
             const int k = min(F - 1, k0 + mt * 16 + h * 8 + g);    // rows past the clip repeat the last frame
             arow[mt][h] = reinterpret_cast<const uint4*>(X + ((size_t)k * N + i) * C);
         }
+    // split K: warp w takes 64-byte blocks w, w + 8, ...; kMmaStages - 1 blocks are in flight per warp
+    const int nblk = (units + 3) / 4;
+    uint4* wring = ring + (size_t)w * kMmaStages * PIECES * 32;
+    const int nmine = nblk > w ? (nblk - w + kMmaWarps - 1) / kMmaWarps : 0;      // blocks of this warp
     const uint4* brow[NT];
     bool bvalid[NT];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) { brow[nt] = nullptr; bvalid[nt] = false; }
+
+    // source rows of the first stages: one copy group, in flight while the anchor is found
+#pragma unroll
+    for (int st = 0; st < kMmaStages - 1; ++st)
+        if (st < nmine)
+            mma_issue_stage<MT, NT, true, false>(wring + st * PIECES * 32, arow, brow, bvalid,
+                                                 (w + st * kMmaWarps) * 4 + tig, units, lane);
+    cp_async_commit();
+
+    const int a = anchor_fn();
+
+    if (tid < NC) s_j[tid] = cand_index(tid);
+    if constexpr (!GRAM) {                       // inverse norms from the sweep's partials
+        const size_t FN = (size_t)F * N;
+        for (int q = tid; q < FR + NC; q += kMmaWarps * 32) {
+            if (q < FR) { const int k = k0 + q; s_rs[q] = k < F ? inv_norm(ssq, nslice, FN, (size_t)k * N + i) : 0.f; }
+            else { const int j = cand_index(q - FR); s_ra[q - FR] = j >= 0 ? inv_norm(ssq, nslice, FN, (size_t)a * N + j) : 0.f; }
+        }
+    }
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
         const int j = cand_index(nt * 8 + g);
@@ -188,14 +212,13 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
         for (int nt = 0; nt < (GRAM ? NT : 1); ++nt) accb[nt][q] = 0.f;
     }
 
-    // split K: warp w takes 64-byte blocks w, w + 8, ...; kMmaStages - 1 blocks are in flight per warp
-    const int nblk = (units + 3) / 4;
-    uint4* wring = ring + (size_t)w * kMmaStages * PIECES * 32;
-    const int nmine = nblk > w ? (nblk - w + kMmaWarps - 1) / kMmaWarps : 0;      // blocks of this warp
+    // candidate rows of the first stages, one copy group per stage.  Groups so far: the source-row group, then
+    // these; the main loop adds one group per block, so "all but the newest ST - 1" still means "block b landed".
 #pragma unroll
     for (int st = 0; st < kMmaStages - 1; ++st) {
         if (st < nmine)
-            mma_issue_stage<MT, NT>(wring + st * PIECES * 32, arow, brow, bvalid, (w + st * kMmaWarps) * 4 + tig, units, lane);
+            mma_issue_stage<MT, NT, false, true>(wring + st * PIECES * 32, arow, brow, bvalid,
+                                                 (w + st * kMmaWarps) * 4 + tig, units, lane);
         cp_async_commit();
     }
     for (int b = 0; b < nmine; ++b) {
