@@ -10,7 +10,10 @@ constexpr int kCopyWarps = 8;
 constexpr int kScanChunks = 4;       // frame counts per lane fetched at once by the warp-level frame search
 
 // Tokens fused into each anchor cell j: |{(k,i): k != a, keep = 0, dst = j}|, gather-side (every cell looks at
-// the (2r+1)^2 x (F-1) tokens that can point to it), integer, fixed order.  Run by whole CTAs: block `b` of `nb`.
+// the (2r+1)^2 x (F-1) tokens that can point to it), integer, order-free.  Run by whole CTAs: block `b` of `nb`,
+// one warp per cell.  The lanes split the (frame, window cell) pairs of the cell and fetch both flags of four
+// pairs at a time without testing one before loading the other, so the loads of a lane overlap instead of
+// forming a chain of dependent round trips.
 __device__ __forceinline__ void fuse_count_cta(int F, int H, int W, int r, int a, const unsigned char* keep,
                                                const int* dst, int* fuse_cnt, int b, int nb) {
     if (fuse_cnt == nullptr) return;
@@ -18,14 +21,24 @@ __device__ __forceinline__ void fuse_count_cta(int F, int H, int W, int r, int a
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     for (int j = b * kCopyWarps + w; j < N; j += nb * kCopyWarps) {
         const int y = j / W, x = j - y * W;
+        const int y_lo = max(0, y - r), x_lo = max(0, x - r);
+        const int nx = min(W - 1, x + r) - x_lo + 1, wsz = (min(H - 1, y + r) - y_lo + 1) * nx;
+        const long long pairs = (long long)F * wsz;
         int c = 0;
-        for (int k = lane; k < F; k += 32) {
-            if (k == a) continue;
-            for (int yy = max(0, y - r); yy <= min(H - 1, y + r); ++yy)
-                for (int xx = max(0, x - r); xx <= min(W - 1, x + r); ++xx) {
-                    const size_t f = (size_t)k * N + yy * W + xx;
-                    c += (!__ldcg(keep + f) && __ldcg(dst + f) == j) ? 1 : 0;
-                }
+        for (long long q0 = lane; q0 < pairs; q0 += 4 * 32) {
+            unsigned char kp[4];
+            int ds[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const long long q = q0 + u * 32;
+                const int k = (int)(q / wsz), e = (int)(q - (long long)k * wsz);
+                const bool in = q < pairs && k != a;
+                const size_t f = (size_t)k * N + (y_lo + e / nx) * W + x_lo + e % nx;
+                kp[u] = in ? __ldcg(keep + f) : (unsigned char)1;
+                ds[u] = in ? __ldcg(dst + f) : -1;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) c += (!kp[u] && ds[u] == j) ? 1 : 0;
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
