@@ -414,7 +414,7 @@ def main():
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(spec, t, nclips, "4 (library: ttf_compress_batch)" if args.streams == 0 else nstreams,
+            "config": workload_config(spec, t, nclips, "8 (library: ttf_compress_batch)" if args.streams == 0 else nstreams,
                                       tokens_step, args.anchor, use_graph),
             "clips_per_s": clips_per_s, "rho": rho, "count_mean": avg_count,
             "roofline": roofline, "pass_roofline": pass_roofline, "cpu_baseline": cpu, "e2e": e2e,

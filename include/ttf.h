@@ -93,10 +93,10 @@ int ttf_compress(const void* features, int F, int H, int W, int C, int r, float 
  * A batch of clips of one shape in one call (the long-video workload: the clips of a request processed
  * concurrently; Sec. 3 treats every clip independently, so this is scheduling only and each clip's results are
  * exactly those of ttf_compress).  features, out_tokens, out_count and out_pos_thw are HOST arrays of nclips
- * DEVICE pointers, read before the call returns.  The clips are spread round-robin over four streams that the
+ * DEVICE pointers, read before the call returns.  The clips are spread round-robin over eight streams that the
  * library keeps per device; these fork from `stream` and join it again through events, so the call is
  * asynchronous, ordered on `stream` like any other, and can be captured in a CUDA graph.  The kernels of one clip
- * leave much of the GPU idle while they ramp up and drain; with four clips in flight those gaps are filled.
+ * leave much of the GPU idle while they ramp up and drain; with several clips in flight those gaps are filled.
  * Scratch: one block per internal stream, from the cache.
  * With the single-launch pass switched on (ttf_set_single_launch) qualifying batches instead run as one persistent
  * cooperative launch per 32 clips in which two groups of CTAs work on consecutive clips half a clip apart.

@@ -421,7 +421,7 @@ int ttf_compress_mean(const void* features, int F, int H, int W, int C, int r, f
 // The clips of a batch are independent, and the kernels of one clip leave most of the GPU idle while they ramp up
 // and drain, so a batch is spread round-robin over kBatchStreams internal streams per device that fork from the
 // caller's stream and join it again (events only: the call stays asynchronous and can be captured in a graph).
-constexpr int kBatchStreams = 4;
+constexpr int kBatchStreams = 8;
 struct BatchLanes { cudaStream_t s[kBatchStreams] = {}; cudaEvent_t fork = nullptr; cudaEvent_t join[kBatchStreams] = {}; bool ok = false; };
 static std::map<int, BatchLanes> g_lanes;
 

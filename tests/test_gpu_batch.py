@@ -32,7 +32,7 @@ def single_launch():
 
 def test_batch_on_library_streams_matches_single_calls_and_oracle():
     s = clips.CONFIGS["vl2b_cal"]
-    Xn = [clips.make_clip(s, s.seed + j) for j in range(7)]          # 7 clips over 4 streams: ragged last round
+    Xn = [clips.make_clip(s, s.seed + j) for j in range(11)]         # 11 clips over 8 streams: ragged last round
     Xs = [to_device(x) for x in Xn]
     outs = P.ttf_compress_batch(Xs, s.r, s.t)
     torch.cuda.synchronize()
