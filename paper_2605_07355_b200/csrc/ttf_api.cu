@@ -424,6 +424,7 @@ int ttf_compress_mean(const void* features, int F, int H, int W, int C, int r, f
 constexpr int kBatchStreams = 8;
 struct BatchLanes { cudaStream_t s[kBatchStreams] = {}; cudaEvent_t fork = nullptr; cudaEvent_t join[kBatchStreams] = {}; bool ok = false; };
 static std::map<int, BatchLanes> g_lanes;
+static std::mutex g_lane_mu;                     // the fork / join events are shared: one batch is enqueued at a time
 
 static int batch_lanes(BatchLanes** out) {
     int dev = 0;
@@ -447,6 +448,7 @@ static int batch_lanes(BatchLanes** out) {
 static int batch_on_streams(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
                             int dtype, void* const* out_tokens, int* const* out_count, int* const* out_pos_thw,
                             cudaStream_t st) {
+    std::lock_guard<std::mutex> enqueue(g_lane_mu);
     BatchLanes* L = nullptr;
     int rc = batch_lanes(&L);
     if (rc != TTF_OK) return rc;
