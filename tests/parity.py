@@ -1,6 +1,6 @@
 """Element-by-element comparison of the CUDA library (through its C ABI) with the CPU oracle.
 
-Tolerances (derived in the design doc):
+Tolerances:
   * anchor index, dst, keep, fuse counts, L', positions, token rows: bit-exact, except
       - keep may differ only where the oracle's fp32-rounded similarity lies within BAND of t,
       - dst may differ only where the oracle's best and second-best similarity are within BAND;
