@@ -143,3 +143,34 @@ def test_bench_configuration_full_size_against_oracle():
         assert (to_bits(toks[j][:L]) == forced.tokens).all()
         rhos.append(1.0 - L / s.tokens)
     assert abs(float(np.mean(rhos)) - 0.67) < 0.03
+
+
+def test_single_launch_batch_longer_than_one_launch():
+    """more clips than one cooperative launch takes (32): the batch is cut into launches that reuse the scratch"""
+    Xs = [to_device(corr_clip(3, 4, 4, 64, seed=100 + j, dtype="bf16")) for j in range(35)]
+    ref = [P.ttf_compress(x, 1, 0.7) for x in Xs]
+    torch.cuda.synchronize()
+    before = P.ttf_set_single_launch(True)
+    try:
+        toks, cnts, poss = P.ttf_compress_batch(Xs, 1, 0.7)
+        torch.cuda.synchronize()
+    finally:
+        P.ttf_set_single_launch(before)
+    for j in range(len(Xs)):
+        L = int(ref[j][1].item())
+        assert int(cnts[j].item()) == L
+        assert torch.equal(toks[j][:L], ref[j][0][:L]) and torch.equal(poss[j][:L], ref[j][2][:L])
+
+
+def test_host_batch_fp32_and_single_clip():
+    Xn = [corr_clip(4, 3, 5, 24, seed=70 + j, dtype="f32") for j in range(3)]
+    host = [torch.from_numpy(x) for x in Xn]                              # pageable memory works too
+    toks, Ls, poss = P.ttf_compress_host_batch(host, 1, 0.6)
+    for j, x in enumerate(Xn):
+        R = O.compress(x, 1, 0.6)
+        q = P.ttf_query(to_device(x), 1, 0.6)
+        forced = O.compress(x, 1, 0.6, anchor_frame=int(q["anchor"].item()), forced_keep=q["keep"].cpu().numpy())
+        assert Ls[j] == forced.count
+        assert (toks[j].numpy() == forced.tokens).all() and (poss[j].numpy() == forced.pos).all()
+    one = P.ttf_compress_host_batch(host[:1], 1, 0.6)
+    assert one[1][0] == Ls[0] and torch.equal(one[0][0], toks[0])

@@ -80,3 +80,17 @@ def test_mean_fuse_paper_shaped(name):
     s = clips.CONFIGS[name]
     fused = check_mean(clips.make_clip(s), s.r, s.t)
     assert fused > 0.4 * s.tokens
+
+
+def test_mean_fuse_misaligned_base_pointer_takes_scalar_path():
+    F, H, W, C = 4, 4, 5, 64
+    X = corr_clip(F, H, W, C, seed=15, dtype="bf16")
+    buf = torch.zeros(F * H * W * C + 8, dtype=torch.bfloat16, device="cuda")
+    view = buf[1:1 + F * H * W * C].view(F, H, W, C)                  # 2 bytes off a 16-byte boundary
+    view.copy_(to_device(X))
+    assert view.data_ptr() % 16 != 0
+    a = P.ttf_compress_mean(view, 1, 0.6)
+    b = P.ttf_compress_mean(to_device(X), 1, 0.6)
+    torch.cuda.synchronize()
+    L = int(a[1].item())
+    assert L == int(b[1].item()) and torch.equal(a[0][:L], b[0][:L]) and torch.equal(a[2][:L], b[2][:L])
