@@ -184,3 +184,34 @@ def test_many_frames_uses_prescanned_prefix():
     X = corr_clip(F, H, W, C, seed=77, dtype="bf16", sigma=0.8)
     rep = check_clip(X, 1, 0.7)
     assert 4 < rep["count"] < F * 4
+
+
+@pytest.mark.parametrize("dtype,C", [("bf16", 256), ("f32", 40)])
+def test_non_finite_tokens_are_kept(dtype, C):
+    """a NaN similarity keeps the token (the gate is evaluated as !(s_hat > t)); other tokens are unaffected"""
+    F, H, W = 5, 6, 7
+    N = H * W
+    Xf = corr_clip(F, H, W, C, seed=91, dtype="f32")
+    Xf[0, 1, 1, 5] = np.nan            # a source token
+    Xf[2, 3, 3, 7] = np.nan            # a token of the anchor frame (frame 2 below)
+    Xf[4, 2, 2, 0] = np.inf            # an infinite source token: its norm is infinite, the cosine NaN
+    X = Xf if dtype == "f32" else clips.f32_to_bf16_bits(Xf)
+    Xd = to_device(X)
+    R = O.compress(X, 1, 0.6, anchor_frame=2)
+    q = P.ttf_query(Xd, 1, 0.6, anchor_mode=3, anchor_frame=2)
+    toks, cnt, pos = P.ttf_compress(Xd, 1, 0.6, anchor_mode=3, anchor_frame=2)
+    torch.cuda.synchronize()
+    keep = q["keep"].cpu().numpy()
+    sim = q["best_sim"].cpu().numpy()
+    assert keep[0 * N + 1 * W + 1] == 1 and keep[4 * N + 2 * W + 2] == 1
+    assert np.isnan(sim[0 * N + 1 * W + 1]) and np.isnan(R.s_hat[0 * N + 1 * W + 1])
+    finite = np.isfinite(R.s_hat)
+    assert (np.isfinite(sim) == finite).all()
+    assert np.abs(sim[finite] - R.s_hat[finite]).max() <= 2e-5
+    in_band = finite & (np.abs(R.s_hat.astype(np.float32) - np.float32(0.6)) < 1e-4)
+    assert not ((keep != R.keep) & ~in_band).any()
+    forced = O.compress(X, 1, 0.6, anchor_frame=2, forced_keep=keep)
+    L = int(cnt.item())
+    assert L == forced.count and (pos[:L].cpu().numpy() == forced.pos).all()
+    bits = (lambda v: v.view(np.uint32)) if dtype == "f32" else (lambda v: v)     # NaN rows compare by bit pattern
+    assert (bits(to_bits(toks[:L])) == bits(np.ascontiguousarray(forced.tokens))).all()
