@@ -97,7 +97,8 @@ int ttf_compress(const void* features, int F, int H, int W, int C, int r, float 
  * library keeps per device; these fork from `stream` and join it again through events, so the call is
  * asynchronous, ordered on `stream` like any other, and can be captured in a CUDA graph.  The kernels of one clip
  * leave much of the GPU idle while they ramp up and drain; with several clips in flight those gaps are filled.
- * Scratch: one block per internal stream, from the cache.
+ * Scratch: one block per internal stream, from the cache.  The streams, their events and the scratch are created by
+ * the first call on a device: make that call outside any stream capture.
  * With the single-launch pass switched on (ttf_set_single_launch) qualifying batches instead run as one persistent
  * cooperative launch per 32 clips in which two groups of CTAs work on consecutive clips half a clip apart.
  */
