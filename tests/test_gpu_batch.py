@@ -174,3 +174,27 @@ def test_host_batch_fp32_and_single_clip():
         assert (toks[j].numpy() == forced.tokens).all() and (poss[j].numpy() == forced.pos).all()
     one = P.ttf_compress_host_batch(host[:1], 1, 0.6)
     assert one[1][0] == Ls[0] and torch.equal(one[0][0], toks[0])
+
+
+def test_long_video_batch_of_eight_against_oracle():
+    """the long-video configuration at full size: 8 clips of F=128 frames in one ttf_compress_batch call"""
+    s = clips.CONFIGS["long_cal"]
+    n = 8
+    Xs, refs = [], []
+    for j in range(n):
+        Xn = clips.make_clip(s, s.seed + j)
+        refs.append((Xn, O.compress(Xn, s.r, s.t)))
+        Xs.append(to_device(Xn))
+    toks, cnts, poss = P.ttf_compress_batch(Xs, s.r, s.t)
+    torch.cuda.synchronize()
+    for j, (Xn, R) in enumerate(refs):
+        q = P.ttf_query(Xs[j], s.r, s.t)
+        keep = q["keep"].cpu().numpy()
+        assert int(q["anchor"].item()) == R.anchor
+        in_band = np.abs(R.s_hat.astype(np.float32) - np.float32(s.t)) < 1e-4
+        assert not ((keep != R.keep) & ~in_band).any()
+        forced = O.compress(Xn, s.r, s.t, anchor_frame=R.anchor, forced_keep=keep)
+        L = int(cnts[j].item())
+        assert L == forced.count
+        assert (poss[j][:L].cpu().numpy() == forced.pos).all()
+        assert (to_bits(toks[j][:L]) == forced.tokens).all()
