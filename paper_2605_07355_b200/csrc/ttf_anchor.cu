@@ -1,5 +1,5 @@
 // Anchor Frame Selection (Eq. auto_anchor) and per-token norms: one streaming sweep over X plus a small
-// statistics kernel; the arg max itself is taken by the matching kernel's prologue (resolve_anchor).
+// statistics kernel whose last CTA takes the arg max (resolve_anchor).
 //
 // k_norm_sum.  A CTA owns (frame k, channel slice q); a slice is LS = 32 lanes x one 16-byte load (512 bytes
 // of every token row; the CTAs of neighbouring slices run side by side, so DRAM sees whole rows).  The
@@ -170,7 +170,7 @@ constexpr int kStatSub = 1;
 
 template <int V>
 __global__ void __launch_bounds__(kNormThreads)
-k_frame_stats(const float* S, int F, int C, int nsl, float* Dp, float* Qp, float* Gp, int* hdr)
+k_frame_stats(const float* S, int F, int C, int nsl, float* Dp, float* Qp, float* Gp, int* hdr, int* out_anchor)
 {
     pdl_launch_dependents();
     trace_mark(hdr, 1, false);
@@ -252,18 +252,30 @@ k_frame_stats(const float* S, int F, int C, int nsl, float* Dp, float* Qp, float
         gg = warp_sum(gg);
         if (lane < kStatReplicas) Gp[(size_t)lane * nsl + q] = gg;
     }
-    trace_mark(hdr, 1, true);
-}
 
-// Clips with more frames than the matching kernel resolves by itself: one CTA takes the arg max.
-__global__ void __launch_bounds__(kNormThreads)
-k_anchor_final(AnchorSrc src, int F)
-{
-    const int a = resolve_anchor(src, F);
-    if (threadIdx.x == 0) {
-        src.hdr[HDR_ANCHOR] = a;
-        if (src.out_anchor) *src.out_anchor = a;
+    // The CTA that finishes last takes the arg max over the frames (Eq. auto_anchor) for the whole clip, so that the
+    // CTAs of the matching kernel only read one word instead of each repeating the search while they hold most of an
+    // SM.  The arrival counter is left at zero for the next call.
+    __shared__ int s_last;
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        s_last = atomicAdd(hdr + HDR_DONE_ALL, 1) == (int)gridDim.x - 1;
     }
+    __syncthreads();
+    if (s_last) {
+        __threadfence();
+        AnchorSrc src;
+        src.Dp = Dp; src.Qp = Qp; src.Gp = Gp; src.nsl = nsl; src.fixed = -1; src.from_hdr = 0; src.hdr = hdr;
+        src.out_anchor = out_anchor;
+        const int a = resolve_anchor(src, F);
+        if (tid == 0) {
+            hdr[HDR_ANCHOR] = a;
+            if (out_anchor) *out_anchor = a;
+            hdr[HDR_DONE_ALL] = 0;
+        }
+    }
+    trace_mark(hdr, 1, true);
 }
 
 cudaError_t launch_norm_sum(const Problem& p, const Scratch& s, cudaStream_t st) {
@@ -273,21 +285,11 @@ cudaError_t launch_norm_sum(const Problem& p, const Scratch& s, cudaStream_t st)
 
 cudaError_t launch_frame_stats(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st) {
     if (p.anchor_mode != 0) return cudaSuccess;                // fixed anchors need no statistics
-    cudaError_t e;
     if (p.C % 4 == 0)
-        e = launch_pdl(k_frame_stats<4>, dim3(p.nsl), dim3(kNormThreads), st, (const float*)s.S, p.F, p.C, p.nsl,
-                       s.Dp, s.Qp, s.Gp, s.hdr);
-    else
-        e = launch_pdl(k_frame_stats<1>, dim3(p.nsl), dim3(kNormThreads), st, (const float*)s.S, p.F, p.C, p.nsl,
-                       s.Dp, s.Qp, s.Gp, s.hdr);
-    if (e != cudaSuccess) return e;
-    if (p.F > kResolveMaxF) {
-        AnchorSrc src = make_anchor_src(p, s, out_anchor);
-        src.from_hdr = 0;
-        k_anchor_final<<<1, kNormThreads, 0, st>>>(src, p.F);
-        e = cudaGetLastError();
-    }
-    return e;
+        return launch_pdl(k_frame_stats<4>, dim3(p.nsl), dim3(kNormThreads), st, (const float*)s.S, p.F, p.C, p.nsl,
+                          s.Dp, s.Qp, s.Gp, s.hdr, out_anchor);
+    return launch_pdl(k_frame_stats<1>, dim3(p.nsl), dim3(kNormThreads), st, (const float*)s.S, p.F, p.C, p.nsl,
+                      s.Dp, s.Qp, s.Gp, s.hdr, out_anchor);
 }
 
 }  // namespace ttf

@@ -14,7 +14,7 @@ constexpr int kHdrInts = 64;
 constexpr int kStatReplicas = 16;      // copies of the frame statistics, so that the CTAs that read them at the
                                        // same moment do not all queue on the same few cache lines
 constexpr int kFusedMaxSplit = 4;     // fused pass: at most this many token ranges per frame in the sweep
-constexpr int kResolveMaxF = 256;      // clips up to this many frames: the matching kernel takes the arg max itself
+constexpr int kResolveMaxF = 256;      // single-launch pass: clips up to this many frames (every CTA takes the arg max itself)
 
 // header words of the scratch block
 enum { HDR_ANCHOR = 0, HDR_DONE_ALL = 1, HDR_ERROR = 2,     // HDR_ERROR: a bounded wait gave up
@@ -121,7 +121,7 @@ inline AnchorSrc make_anchor_src(const Problem& p, const Scratch& s, int* out_an
     AnchorSrc a;
     a.Dp = s.Dp; a.Qp = s.Qp; a.Gp = s.Gp; a.nsl = p.nsl; a.hdr = s.hdr; a.out_anchor = out_anchor;
     a.fixed = p.anchor_mode == 0 ? -1 : (p.anchor_mode == 1 ? 0 : (p.anchor_mode == 2 ? p.F - 1 : p.anchor_arg));
-    a.from_hdr = (p.anchor_mode == 0 && p.F > kResolveMaxF) ? 1 : 0;
+    a.from_hdr = p.anchor_mode == 0 ? 1 : 0;     // the statistics kernel's last CTA left the arg max there
     return a;
 }
 
