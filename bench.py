@@ -56,8 +56,8 @@ def parse_args():
 
 # DRAM bytes (read + write) per launch from the committed ncu capture (profiles/kernels_full_vl8b_cal.md: cold
 # caches, one launch of each kernel).  Valid only for the kernels as captured; other workloads report null.
-NCU_TRAFFIC = {("vl8b_cal", "match"): 67275520 + 928768, ("vl8b_cal", "norm_sum"): 67120384 + 476928,
-               ("vl8b_cal", "compact"): 24694016 + 43776}
+NCU_TRAFFIC = {("vl8b_cal", "match"): 67141888 + 1333248, ("vl8b_cal", "norm_sum"): 67120128 + 563968,
+               ("vl8b_cal", "compact"): 24693760 + 80896}
 
 
 def peaks():
