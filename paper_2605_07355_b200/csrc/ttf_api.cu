@@ -147,6 +147,14 @@ static int clear_control(const Problem&, void* ws, cudaStream_t st) {
     return e == cudaSuccess ? TTF_OK : cuda_fail(e);
 }
 
+// The control words of `n` scratch blocks `stride` bytes apart.  A cached allocation that is reused with another
+// clip shape holds old data where the new layout has its control words; block 0 of the cache is kept clean by the
+// kernels themselves, the further blocks of a multi-clip layout are cleared before use.
+static int clear_control_blocks(void* ws, size_t stride, int n, cudaStream_t st) {
+    cudaError_t e = cudaMemset2DAsync(ws, stride, 0, sizeof(int) * kHdrInts, (size_t)n, st);
+    return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+}
+
 // steps shared by compress and query: norms + frame sums, anchor, matching + gate
 static int run_front(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                      unsigned char* keep, cudaStream_t st) {
@@ -497,6 +505,8 @@ int ttf_compress_batch(const void* const* features, int nclips, int F, int H, in
     void* ws = nullptr;
     rc = cached_scratch(stride * chunk, st, &ws);
     if (rc != TTF_OK) return rc;
+    rc = clear_control_blocks(ws, stride, chunk, st);
+    if (rc != TTF_OK) return rc;
     carve_scratch(p, ws, &s);
     for (int base = 0; base < nclips; base += kFusedBatchMax) {
         const int m = nclips - base < kFusedBatchMax ? nclips - base : kFusedBatchMax;
@@ -763,6 +773,8 @@ int ttf_profile_stages(const void* const* features, int nclips, int F, int H, in
     }
     void* ws = nullptr;
     int rc = cached_scratch(stride * nclips, st, &ws);
+    if (rc != TTF_OK) return rc;
+    rc = clear_control_blocks(ws, stride, nclips, st);
     if (rc != TTF_OK) return rc;
     cudaEvent_t ev[5];
     for (auto& e : ev) if (cudaEventCreate(&e) != cudaSuccess) return cuda_fail(cudaGetLastError());

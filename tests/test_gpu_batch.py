@@ -198,3 +198,24 @@ def test_long_video_batch_of_eight_against_oracle():
         assert L == forced.count
         assert (poss[j][:L].cpu().numpy() == forced.pos).all()
         assert (to_bits(toks[j][:L]) == forced.tokens).all()
+
+
+def test_multi_block_scratch_after_another_shape_on_the_same_stream():
+    """the per-stream scratch cache is reused with another layout: blocks of the batch land on old data"""
+    st = torch.cuda.Stream()
+    big = to_device(clips.make_clip(clips.CONFIGS["vl2b_cal"]))
+    small = [to_device(corr_clip(4, 5, 5, 128, seed=200 + j, dtype="bf16")) for j in range(6)]
+    ref = [P.ttf_compress(x, 1, 0.7) for x in small]
+    torch.cuda.synchronize()
+    with torch.cuda.stream(st):
+        P.ttf_compress(big, 1, 0.7, stream=st)                     # fills the stream's scratch with its arrays
+        before = P.ttf_set_single_launch(True)
+        try:
+            toks, cnts, poss = P.ttf_compress_batch(small, 1, 0.7, stream=st)
+        finally:
+            P.ttf_set_single_launch(before)
+    st.synchronize()
+    for j in range(len(small)):
+        L = int(ref[j][1].item())
+        assert int(cnts[j].item()) == L
+        assert torch.equal(toks[j][:L], ref[j][0][:L]) and torch.equal(poss[j][:L], ref[j][2][:L])
