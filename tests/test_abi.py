@@ -69,6 +69,31 @@ def test_null_and_nonfinite_arguments_are_rejected_before_any_launch(lib):
     assert lib.ttf_query_ex(fake, 4, 4, 4, 8, 1, 0.7, 0, 3, -1, None, None, None, None, None, None) == 1
 
 
+def test_batch_and_variant_entry_points_validate_before_any_cuda_call(lib):
+    fake = ctypes.c_void_p(4096)
+    arr = (ctypes.c_void_p * 2)(4096, 8192)
+    hole = (ctypes.c_void_p * 2)(4096, None)
+    counts = (ctypes.c_int * 2)()
+    f = lib.ttf_compress_batch
+    assert f(None, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, None) == 1
+    assert f(arr, 0, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, None) == 1
+    assert f(hole, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, None) == 1          # a NULL clip inside the batch
+    assert f(arr, 2, 4, 4, 4, 0, 1, 0.7, 0, arr, arr, arr, None) == 1
+    assert f(arr, 2, 4, 4, 4, 8, 1, float("nan"), 0, arr, arr, arr, None) == 1
+    h = lib.ttf_compress_host_batch
+    assert h(arr, 0, 4, 4, 4, 8, 1, 0.7, 0, arr, ctypes.cast(counts, ctypes.c_void_p), arr) == 1
+    assert h(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, hole, ctypes.cast(counts, ctypes.c_void_p), arr) == 1
+    assert h(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, None, arr) == 1
+    assert h(arr, 2, 4, 4, 4, 8, -1, 0.7, 0, arr, ctypes.cast(counts, ctypes.c_void_p), arr) == 1
+    assert lib.ttf_compress_mean(None, 4, 4, 4, 8, 1, 0.7, 0, fake, fake, fake, None) == 1
+    assert lib.ttf_compress_mean(fake, 4, 4, 4, 8, 1, 0.7, 2, fake, fake, fake, None) == 1
+    ms = (ctypes.c_double * 6)()
+    assert lib.ttf_profile_stages(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, 0, ms, 6, None) == 1   # reps < 1
+    assert lib.ttf_profile_stages(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, 1, None, 6, None) == 1
+    before = lib.ttf_set_single_launch(1)
+    assert lib.ttf_set_single_launch(before) == 1 and lib.ttf_set_single_launch(before) == before
+
+
 def test_decode_alignment_helper():
     assert P.ttf_decode_pos(2703, 57, 0) == 2760 and P.ttf_decode_pos(2703, 57, 4) == 2764
 
