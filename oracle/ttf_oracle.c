@@ -243,21 +243,17 @@ void ttf_oracle_restore(const void* compressed, size_t row_bytes, const uint8_t*
 
 /*
  * Distribution of the best-match similarities of the source tokens (Discussion D1): counts over `bins` equal
- * bins of [-1, 1], bin = floor((s + 1) / 2 * bins) evaluated in fp32 like the CUDA path, clamped; NaN skipped.
+ * bins of [-1, 1]: bin = floor((s + 1) / 2 * bins), clamped to [0, bins - 1]; NaN skipped.  Plain double.
  */
 void ttf_oracle_sim_histogram(const float* s_hat, int F, int N, int a, int bins, unsigned int* hist) {
     for (int b = 0; b < bins; ++b) hist[b] = 0;
     for (int k = 0; k < F; ++k) {
         if (k == a) continue;
         for (int i = 0; i < N; ++i) {
-            float s = s_hat[(size_t)k * N + i];
+            double s = (double)s_hat[(size_t)k * N + i];
             if (!(s == s)) continue;
-            volatile float u = s + 1.0f;            /* keep every step in fp32 */
-            volatile float v = u * 0.5f;
-            volatile float x = v * (float)bins;
-            int b = (int)floorf(x);
-            if (b < 0) b = 0;
-            if (b >= bins) b = bins - 1;
+            double x = floor((s + 1.0) / 2.0 * (double)bins);
+            int b = x < 0.0 ? 0 : (x >= (double)bins ? bins - 1 : (int)x);
             hist[b] += 1;
         }
     }

@@ -176,9 +176,12 @@ def test_host_batch_fp32_and_single_clip():
     assert one[1][0] == Ls[0] and torch.equal(one[0][0], toks[0])
 
 
-def test_long_video_batch_of_eight_against_oracle():
-    """the long-video configuration at full size: 8 clips of F=128 frames in one ttf_compress_batch call"""
-    s = clips.CONFIGS["long_cal"]
+@pytest.mark.parametrize("name", ["long", "long_cal"])
+def test_long_video_batch_of_eight_against_oracle(name):
+    """the long-video configuration at full size: 8 clips of F=128 frames in one ttf_compress_batch call; `long`
+    is the configuration text word for word (per-clip noise level, Poisson scene cuts), `long_cal` the anchored
+    variant the throughput runs use"""
+    s = clips.CONFIGS[name]
     n = 8
     Xs, refs = [], []
     for j in range(n):

@@ -45,9 +45,20 @@ def test_histogram_matches_oracle(bins):
     q = P.ttf_query(Xd, s.r, s.t)
     hist = P.ttf_sim_histogram(q["best_sim"], q["anchor"], s.F, s.H, s.W, bins)
     torch.cuda.synchronize()
-    ref = O.sim_histogram(q["best_sim"].cpu().numpy(), s.F, s.N, int(q["anchor"].item()), bins)
-    got = hist.cpu().numpy().view(np.uint32)
-    assert (got == ref).all() and got.sum() == (s.F - 1) * s.N
+    sim = q["best_sim"].cpu().numpy()
+    a = int(q["anchor"].item())
+    ref = O.sim_histogram(sim, s.F, s.N, a, bins).astype(np.int64)
+    got = hist.cpu().numpy().view(np.uint32).astype(np.int64)
+    assert got.sum() == (s.F - 1) * s.N
+    # the oracle bins in double, the kernel in fp32: a similarity within 1e-6 of a bin edge may land on either
+    # side of it.  Such values are counted per edge; every other value must be in the oracle's bin.
+    src = np.delete(sim.reshape(s.F, s.N), a, axis=0).ravel().astype(np.float64)
+    x = (src + 1.0) / 2.0 * bins
+    e = np.rint(x)
+    near = (np.abs(x - e) * 2.0 / bins < 1e-6) & (e >= 1) & (e <= bins - 1)
+    slack = np.bincount(e[near].astype(np.int64), minlength=bins + 1)      # slack[j]: values near the edge below bin j
+    print(f"bins={bins}: {int(near.sum())} similarities within 1e-6 of a bin edge")
+    assert (np.abs(got - ref) <= slack[:bins] + slack[1:bins + 1]).all()
 
 
 @pytest.mark.parametrize("shape,dtype", [((4, 6, 5, 64), "bf16"), ((5, 3, 7, 40), "f32"), ((9, 16, 16, 512), "bf16")])

@@ -103,10 +103,13 @@ def test_paper_shaped_clips(name):
         assert abs(check_clip(X, s.r, 0.70)["rho"] - 0.67) < 0.02
 
 
-def test_wide_search_clip():
-    s = clips.CONFIGS["wide_cal"]
+@pytest.mark.parametrize("name", ["wide", "wide_cal"])
+def test_wide_search_clip(name):
+    """F=64, 32x32, r=2: the configuration text word for word (shifts in {-2..2}^2, outlier tokens) and the
+    anchored variant the throughput runs use"""
+    s = clips.CONFIGS[name]
     rep = check_clip(clips.make_clip(s), s.r, s.t)
-    print(rep)
+    print(name, rep)
 
 
 def test_long_clip_batch_on_streams():

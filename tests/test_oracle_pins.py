@@ -291,6 +291,20 @@ def test_restore_inverts_compaction():
     assert (full3.reshape(3, N, C) == Xi.reshape(3, N, C)).all()
 
 
+def test_fuse_count_is_a_bincount_of_the_fused_destinations():
+    """the bookkeeping of identity replacement written with numpy's own counting routine"""
+    for seed, r, t in [(91, 1, 0.70), (92, 2, 0.5), (93, 0, 0.3)]:
+        F, H, W, C = 6, 5, 7, 32
+        N = H * W
+        R = O.compress(corr_clip(F, H, W, C, seed=seed), r, t)
+        src = np.ones(F * N, dtype=bool)
+        src[R.anchor * N:(R.anchor + 1) * N] = False
+        fused = src & (R.keep == 0)
+        assert fused.any()
+        assert (R.fuse_cnt == np.bincount(R.dst[fused], minlength=N)).all()
+        assert (O.fuse_count(R.keep, R.dst, F, N, R.anchor) == R.fuse_cnt).all()
+
+
 # ---- Discussion D1: distribution of the best similarities ---------------------------------------------------
 @pytest.mark.parametrize("bins", [1, 7, 64, 200])
 def test_sim_histogram_matches_numpy(bins):
@@ -303,8 +317,13 @@ def test_sim_histogram_matches_numpy(bins):
     src = np.delete(s.reshape(F, N), R.anchor, axis=0).ravel()
     ref, _ = np.histogram(src.astype(np.float64), bins=bins, range=(-1.0, 1.0))
     assert h.sum() == (F - 1) * N
-    # numpy bins in float64 with a closed last bin; values on a bin edge may land one bin apart
-    assert np.abs(h.astype(np.int64) - ref).sum() <= 2 and (h.astype(np.int64) == ref).mean() > 0.9
+    # numpy's bins are half-open like the definition except that its last bin is closed, which the clamp reproduces
+    assert (h.astype(np.int64) == ref).all()
+    # values exactly on bin edges, where a wrong rounding direction or a wrong clamp would show
+    edges = np.array([-1.0, -0.5, 0.0, 0.25, 0.5, 1.0, 1.5, -1.5], dtype=np.float32)
+    he = O.sim_histogram(np.concatenate([np.ones(8, np.float32), edges]), 2, 8, 0, 4)      # frame 0 is the anchor
+    # four bins of width 0.5: {-1.5 (clamped), -1} | {-0.5} | {0, 0.25} | {0.5, 1 (closed end), 1.5 (clamped)}
+    assert he.tolist() == [2, 1, 2, 3]
     s2 = s.copy(); s2[N * ((R.anchor + 1) % F)] = np.nan
     assert O.sim_histogram(s2, F, N, R.anchor, bins).sum() == (F - 1) * N - 1
 
