@@ -51,7 +51,8 @@ typedef enum {
     TTF_ERR_UNSUPPORTED = 2,   /* sizes beyond int32 indexing (F*H*W >= 2^31 or F*H*W*C*itemsize >= 2^46)    */
     TTF_ERR_WORKSPACE = 3,     /* caller workspace NULL, smaller than ttf_workspace_bytes or not 256-aligned */
     TTF_ERR_CUDA = 4,          /* a CUDA runtime call failed (see ttf_last_cuda_error)                       */
-    TTF_ERR_STATIC_LIMIT = 5   /* ttf_query_static: the clip needs more scratch than TTF_STATIC_SCRATCH_BYTES */
+    TTF_ERR_TIMEOUT = 5,       /* device status only: a kernel gave up on one of its bounded waits           */
+    TTF_ERR_STATIC_LIMIT = 6   /* ttf_query_static: the clip needs more scratch than TTF_STATIC_SCRATCH_BYTES */
 } ttf_status;
 
 /* anchor rule: Eq. (auto_anchor), or the fixed first / last frame anchors compared in Table 1 and ablation A2,
@@ -67,6 +68,31 @@ const char* ttf_status_string(int status);
 int ttf_last_cuda_error(void);
 
 /*
+ * Device-side status of the most recent call of this library on `stream` (the paper has no counterpart).  The only
+ * waits inside the kernels are waits of a warp for its own asynchronous copies; each is bounded, and a warp whose
+ * wait runs out stops copying and sets an error word in the call's scratch, which the first kernel of every call
+ * clears.  ttf_last_device_status synchronises `stream`, reads the error word(s) of the last call enqueued on it (for
+ * a batch call: of every clip of the batch) and stores TTF_OK or TTF_ERR_TIMEOUT in *host_status.  ttf_compress also
+ * reports the condition as out_count = -1; the query entry points have no other channel than this one.  The return
+ * value is the status of the status query itself.  ttf_workspace_status is the same for calls that ran on
+ * caller-owned scratch (`workspace` as passed to the _ws entry point; NULL = the built-in array of ttf_query_static).
+ */
+int ttf_last_device_status(ttf_stream_t stream, int* host_status);
+int ttf_workspace_status(const void* workspace, ttf_stream_t stream, int* host_status);
+
+/*
+ * Test hooks (the paper has no counterpart; not for production use).
+ * ttf_debug_set_wait: poll_limit = polls of a barrier before a waiting warp gives up (default 2^18); tx_extra_bytes
+ * (a multiple of 16, normally 0) is added to the byte count every copy barrier is told to expect, so that with a
+ * non-zero value the data lands but the barrier never completes and every bounded wait runs out: the give-up path
+ * can be exercised without a fault or a hang.  Process-wide.
+ * ttf_debug_func_attr_needed: the per-(function, device) table behind the kernels' dynamic shared memory limits;
+ * returns 1 when (key, device) had not been recorded with at least `bytes` before, and records it.
+ */
+int ttf_debug_set_wait(int poll_limit, int tx_extra_bytes);
+int ttf_debug_func_attr_needed(const void* key, int device, size_t bytes);
+
+/*
  * Scratch bytes one call needs for a clip of this shape (per-token inverse norms, per-frame channel sums,
  * anchor cosines, s_hat / dst / keep, per-frame survivor counts).  Sec. 3 has no counterpart: this is
  * bookkeeping of the implementation.  The result is a multiple of 256.
@@ -80,7 +106,8 @@ int ttf_workspace_bytes(int F, int H, int W, int C, int r, int dtype, size_t* by
  *                rows [N, N+P) the preserved source tokens in ascending flat index k*N + i (Eq. xprime_stack).
  *   out_count    one int32: L' = N + P (Eq. Lpre).  pos_dec(l) = L' + T + l (Eq. decode_pos) is
  *                ttf_decode_pos below.  -1 reports that a kernel gave up on one of its (bounded) internal
- *                waits, which does not happen on a healthy device; the other outputs are then undefined.
+ *                waits, which does not happen on a healthy device; the other outputs are then undefined
+ *                (see ttf_last_device_status).  It is written last, when every copy has completed.
  *   out_pos_thw  [capacity F*H*W, 3] int32; row j = (k, y, x) of output row j (Eq. compress_pos).
  * Rows beyond L' are not written.  Scratch comes from a cache the library keeps per (device, stream),
  * allocated with cudaMalloc on first use and grown when a larger clip arrives; two calls on the same stream
@@ -99,23 +126,31 @@ int ttf_compress(const void* features, int F, int H, int W, int C, int r, float 
  * leave much of the GPU idle while they ramp up and drain; with several clips in flight those gaps are filled.
  * Scratch: one block per internal stream, from the cache.  The streams, their events and the scratch are created by
  * the first call on a device: make that call outside any stream capture.
- * With the single-launch pass switched on (ttf_set_single_launch) qualifying batches instead run as one persistent
- * cooperative launch per 32 clips in which two groups of CTAs work on consecutive clips half a clip apart.
  */
 int ttf_compress_batch(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
                        int dtype, void* const* out_tokens, int* const* out_count, int* const* out_pos_thw,
                        ttf_stream_t stream);
 
 /*
- * Execution variant (the paper has no counterpart).  on != 0: bf16 clips with r <= 1, 16-byte aligned rows and at
- * most 256 frames run the whole pass as ONE persistent cooperative kernel whose phases are separated by
- * grid-wide barriers (bounded waits; a wait that gives up reports out_count = -1) instead of four kernels.  Results
- * are identical except that the frame sums of Eq. (auto_anchor) are added in a different fixed order.  Off by
- * default (or TTF_SINGLE_LAUNCH=1 in the environment): measured on B200 the kernel sequence is faster for the
- * clip shapes of the paper; the single launch is for callers for whom the number of launches matters.
- * Process-wide; returns the previous setting.
+ * Kernel of the matching step for bf16 clips with r <= 2 and 16-byte aligned rows (the paper has no counterpart; the
+ * results are the same within the stated tolerance): 0 automatic; 1 the warp-level tensor-core MMA kernel (one cell
+ * x 32 frames per CTA, token norms from Gram-tile diagonals); 2 the tcgen05 kernel (strips of 4 cells x 32 frames as
+ * TMA tiles, accumulators in tensor memory, token norms from the sweep; needs C >= 64).  Process-wide; takes effect
+ * with the next call.
  */
-int ttf_set_single_launch(int on);
+int ttf_set_match_kernel(int which);
+
+/*
+ * Schedule of ttf_compress_batch and L2 use of the passes over X (the paper has no counterpart).  Eq. (auto_anchor)
+ * needs all of X before any token can be matched, so X is read twice; the second read is free only for what is still
+ * in L2.  clips_in_flight (0 = automatic, at most 8) bounds how many clips of a batch run concurrently.  l2_mode
+ * selects the L2 eviction priorities the kernels attach to their accesses to X: 0 none; 1 the first
+ * ceil(F * resident_pct / 100) frames of a clip are read with the default priority by the sweep and every other
+ * access (the remaining frames, the matching pass's source rows, the gather's rows and its output) as evict-first;
+ * 2 the same with evict-last for the leading frames.  Results do not depend on any of this.  Process-wide; takes
+ * effect with the next call.
+ */
+int ttf_set_schedule(int clips_in_flight, int l2_mode, int resident_pct);
 
 /* Same, with caller-owned scratch: `workspace` must be 256-byte aligned device memory of at least
  * ttf_workspace_bytes(...) bytes that no other in-flight call uses.  Allocates nothing. */
@@ -255,10 +290,10 @@ int ttf_query_static(const void* features, int F, int H, int W, int C, int r, fl
  * device time in milliseconds and the number of launches; `kinds` is the length of both arrays
  * (TTF_KERNEL_KINDS covers all).  Kinds: 0 frame-sum (and norm) sweep, 1 frame statistics of the anchor rule,
  * 2 windowed match + gate (its prologue takes the anchor arg max), 3 compaction gather (with the frame-count
- * prefix of clips longer than 1024 frames), 4 fuse-count bookkeeping of ttf_query, 5 the single-launch pass.  Profiling is process-wide
+ * prefix of clips longer than 1024 frames), 4 fuse-count bookkeeping of ttf_query.  Profiling is process-wide
  * and meant for benchmarks; leave it off otherwise.
  */
-#define TTF_KERNEL_KINDS 6
+#define TTF_KERNEL_KINDS 5
 int ttf_profile_begin(void);
 int ttf_profile_end(double* total_ms, long long* launches, int kinds);
 
@@ -268,7 +303,7 @@ int ttf_profile_end(double* total_ms, long long* launches, int kinds);
  * own scratch block, with one pair of CUDA events around the group; ms_per_launch[kind] = group time / nclips,
  * averaged over the rounds.  With a batch larger than L2 every launch finds its clip cold in HBM, which is how a
  * kernel runs when several clips are in flight.  Arguments as ttf_compress_batch; the outputs are those of the
- * pass.  Always the kernel sequence, whatever ttf_set_single_launch says.  Synchronises `stream`.
+ * pass.  Synchronises `stream`.
  */
 int ttf_profile_stages(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
                        int dtype, void* const* out_tokens, int* const* out_count, int* const* out_pos_thw,

@@ -22,11 +22,13 @@ EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
     "ttf_query_static", "ttf_compress_ex", "ttf_query_ex", "ttf_compress_segment", "ttf_restore",
-    "ttf_sim_histogram", "ttf_compress_batch", "ttf_set_single_launch", "ttf_profile_stages", "ttf_compress_mean", "ttf_compress_host_batch",
+    "ttf_sim_histogram", "ttf_compress_batch", "ttf_profile_stages", "ttf_compress_mean", "ttf_compress_host_batch",
+    "ttf_set_schedule", "ttf_set_match_kernel", "ttf_last_device_status", "ttf_workspace_status", "ttf_debug_set_wait", "ttf_debug_func_attr_needed",
 ]
+TTF_ERR_TIMEOUT, TTF_ERR_STATIC_LIMIT = 5, 6
 TTF_ANCHOR_AUTO, TTF_ANCHOR_FIRST, TTF_ANCHOR_LAST, TTF_ANCHOR_EXPLICIT = 0, 1, 2, 3
 TTF_STATIC_SCRATCH_BYTES = 8 << 20
-KERNEL_KINDS = ["norm_sum", "frame_stats", "match", "compact", "fuse_count", "single_launch"]
+KERNEL_KINDS = ["norm_sum", "frame_stats", "match", "compact", "fuse_count"]
 
 _lib = None
 
@@ -61,8 +63,18 @@ def lib() -> ctypes.CDLL:
         L.ttf_compress_batch.argtypes = [vp, i] + shape + [f, i, vp, vp, vp, vp]
         L.ttf_profile_stages.restype = i
         L.ttf_profile_stages.argtypes = [vp, i] + shape + [f, i, vp, vp, vp, i, ctypes.POINTER(ctypes.c_double), i, vp]
-        L.ttf_set_single_launch.restype = i
-        L.ttf_set_single_launch.argtypes = [i]
+        L.ttf_last_device_status.restype = i
+        L.ttf_last_device_status.argtypes = [vp, ctypes.POINTER(i)]
+        L.ttf_workspace_status.restype = i
+        L.ttf_workspace_status.argtypes = [vp, vp, ctypes.POINTER(i)]
+        L.ttf_debug_set_wait.restype = i
+        L.ttf_debug_set_wait.argtypes = [i, i]
+        L.ttf_debug_func_attr_needed.restype = i
+        L.ttf_debug_func_attr_needed.argtypes = [vp, i, sz]
+        L.ttf_set_match_kernel.restype = i
+        L.ttf_set_match_kernel.argtypes = [i]
+        L.ttf_set_schedule.restype = i
+        L.ttf_set_schedule.argtypes = [i, i, i]
         L.ttf_compress_mean.restype = i
         L.ttf_compress_mean.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp]
         L.ttf_compress_host_batch.restype = i
@@ -187,9 +199,43 @@ def ttf_profile_stages(features, r: int, t: float, out_tokens, out_count, out_po
     return {k: float(ms[i]) for i, k in enumerate(KERNEL_KINDS[:4])}
 
 
-def ttf_set_single_launch(on: bool) -> bool:
-    """ttf_set_single_launch: switches the one-kernel variant of the pass on or off; returns the previous setting."""
-    return bool(lib().ttf_set_single_launch(1 if on else 0))
+def ttf_last_device_status(stream=None) -> int:
+    """ttf_last_device_status: synchronises the stream; TTF_OK or TTF_ERR_TIMEOUT for the last call on it."""
+    v = ctypes.c_int(0)
+    rc = lib().ttf_last_device_status(_stream_ptr(stream), ctypes.byref(v))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_last_device_status")
+    return int(v.value)
+
+
+def ttf_workspace_status(workspace: Optional[torch.Tensor], stream=None) -> int:
+    """ttf_workspace_status: the same for caller-owned scratch (None = the array of ttf_query_static)."""
+    v = ctypes.c_int(0)
+    rc = lib().ttf_workspace_status(_p(workspace), _stream_ptr(stream), ctypes.byref(v))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_workspace_status")
+    return int(v.value)
+
+
+def ttf_debug_set_wait(poll_limit: int = 1 << 18, tx_extra_bytes: int = 0) -> None:
+    """ttf_debug_set_wait (test hook): poll limit of the bounded waits and extra bytes announced to copy barriers."""
+    rc = lib().ttf_debug_set_wait(int(poll_limit), int(tx_extra_bytes))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_debug_set_wait")
+
+
+def ttf_set_match_kernel(which: int = 0) -> None:
+    """ttf_set_match_kernel: 0 automatic, 1 warp-level MMA kernel, 2 tcgen05 kernel."""
+    rc = lib().ttf_set_match_kernel(int(which))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_set_match_kernel")
+
+
+def ttf_set_schedule(clips_in_flight: int = 0, l2_mode: int = 0, resident_pct: int = 0) -> None:
+    """ttf_set_schedule: clips of a batch in flight (0 = automatic) and the L2 eviction priorities of the passes."""
+    rc = lib().ttf_set_schedule(int(clips_in_flight), int(l2_mode), int(resident_pct))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_set_schedule")
 
 
 def ttf_compress_mean(features: torch.Tensor, r: int, t: float, stream=None):

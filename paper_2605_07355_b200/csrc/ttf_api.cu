@@ -3,6 +3,7 @@
 #include "../../include/ttf.h"
 #include "ttf_internal.cuh"
 
+#include <atomic>
 #include <cmath>
 #include <cstdlib>
 #include <map>
@@ -33,8 +34,42 @@ int sm_count() {
     return n;
 }
 
+// ---- per-(function, device) record of the dynamic shared memory limit that has been set ------------------
+struct FuncAttrTable {
+    std::mutex mu;
+    std::map<std::pair<const void*, int>, size_t> set;
+    // true when (func, dev) has not been given at least `bytes` yet; records it
+    bool needs(const void* func, int dev, size_t bytes) {
+        std::lock_guard<std::mutex> lk(mu);
+        size_t& have = set[std::make_pair(func, dev)];
+        if (have >= bytes) return false;
+        have = bytes;
+        return true;
+    }
+    void forget(const void* func, int dev) {
+        std::lock_guard<std::mutex> lk(mu);
+        set.erase(std::make_pair(func, dev));
+    }
+};
+static FuncAttrTable g_func_attr;
+
+cudaError_t ensure_dynamic_smem(const void* func, size_t bytes) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!g_func_attr.needs(func, dev, bytes)) return cudaSuccess;
+    e = cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) g_func_attr.forget(func, dev);
+    return e;
+}
+
+static std::atomic<int> g_wait_limit{1 << 18};
+static std::atomic<int> g_wait_tx_extra{0};
+int wait_poll_limit() { return g_wait_limit.load(); }
+int wait_tx_extra() { return g_wait_tx_extra.load(); }
+
 // ---- optional per-kernel timing: CUDA events recorded around every launch while profiling is on ---------
-enum { PK_NORM_SUM = 0, PK_FRAME_STATS = 1, PK_MATCH = 2, PK_COMPACT = 3, PK_FUSE_COUNT = 4, PK_FUSED = 5, PK_KINDS = 6 };
+enum { PK_NORM_SUM = 0, PK_FRAME_STATS = 1, PK_MATCH = 2, PK_COMPACT = 3, PK_FUSE_COUNT = 4, PK_KINDS = 5 };
 struct ProfRecord { int kind; cudaEvent_t a, b; };
 static std::mutex g_prof_mu;
 static bool g_prof_on = false;
@@ -55,6 +90,12 @@ struct ProfScope {
     }
 };
 
+// Schedule of a batch: clips in flight and the L2 priorities of the passes over X (ttf_set_schedule)
+static std::atomic<int> g_sched_lanes{0};        // 0: automatic
+static std::atomic<int> g_sched_l2_mode{0};
+static std::atomic<int> g_sched_res_pct{0};
+static std::atomic<int> g_match_kernel{0};       // ttf_set_match_kernel: 0 automatic, 1 warp-level MMA, 2 tcgen05
+
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 void carve_scratch(const Problem& p, void* base, Scratch* s) {
@@ -65,7 +106,7 @@ void carve_scratch(const Problem& p, void* base, Scratch* s) {
     s->hdr = (int*)take(sizeof(int) * kHdrInts);      // control words first: one small memset clears them
     s->cnt = (int*)take(sizeof(int) * p.F);
     s->prefix = (int*)take(sizeof(int) * ((size_t)p.F + 1));
-    s->S = (float*)take(sizeof(float) * (size_t)p.F * p.C * (fused_eligible(p) ? kFusedMaxSplit : 1));
+    s->S = (float*)take(sizeof(float) * (size_t)p.F * p.C);
     s->Dp = (float*)take(sizeof(float) * (size_t)kStatReplicas * p.nsl * p.F);
     s->Qp = (float*)take(sizeof(float) * (size_t)kStatReplicas * p.nsl * p.F);
     s->Gp = (float*)take(sizeof(float) * (size_t)kStatReplicas * p.nsl);
@@ -74,6 +115,9 @@ void carve_scratch(const Problem& p, void* base, Scratch* s) {
     s->dst = (int*)take(sizeof(int) * FN);
     s->keep = (unsigned char*)take(FN);
     s->fuse_cnt = (int*)take(sizeof(int) * p.N);
+    s->tc_tiles = p.use_tc ? (int)tc_match_tiles(p) : 0;
+    s->tc_cnt = (int*)take(sizeof(int) * (size_t)s->tc_tiles);
+    s->tc_part = (float*)take(sizeof(float) * (p.use_tc ? tc_match_part_floats(p) : 0));
     s->bytes = off;
 }
 
@@ -101,11 +145,18 @@ static int make_problem(const void* X, int F, int H, int W, int C, int r, float 
     if ((long long)F * p->nq >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
     p->nsl = C % 4 == 0 ? (C + 127) / 128 : (C + 31) / 32;
     p->anchor_mode = 0; p->anchor_arg = 0; p->emit_anchor = 1; p->pos_t_offset = 0;
+    p->l2_mode = g_sched_l2_mode.load();
+    p->res_frames = (int)(((long long)F * g_sched_res_pct.load() + 99) / 100);
+    p->use_tc = 0;
+    p->use_tc = (g_match_kernel.load() == 2 && tc_match_eligible(*p)) ? 1 : 0;
     return TTF_OK;
 }
 
 // ---- scratch cache: one block per (device, stream), grown on demand -------------------------------------
-struct CacheEntry { void* ptr = nullptr; size_t bytes = 0; };
+struct CacheEntry {
+    void* ptr = nullptr; size_t bytes = 0;
+    std::vector<const int*> status_words;        // header blocks the most recent call on this stream used
+};
 static std::mutex g_mu;
 static std::map<std::pair<int, cudaStream_t>, CacheEntry> g_scratch;
 
@@ -122,6 +173,7 @@ static int cached_scratch(size_t bytes, cudaStream_t st, void** out) {
             if (e != cudaSuccess) return cuda_fail(e);
             cudaFree(ce.ptr);
             ce.ptr = nullptr; ce.bytes = 0;
+            ce.status_words.clear();
         }
         e = cudaMalloc(&ce.ptr, bytes);
         if (e != cudaSuccess) { ce.ptr = nullptr; return cuda_fail(e); }
@@ -131,6 +183,7 @@ static int cached_scratch(size_t bytes, cudaStream_t st, void** out) {
         if (e != cudaSuccess) return cuda_fail(e);
     }
     *out = ce.ptr;
+    ce.status_words.assign(1, reinterpret_cast<const int*>(ce.ptr));
     return TTF_OK;
 }
 
@@ -171,28 +224,10 @@ static int run_front(const Problem& p, const Scratch& s, int* out_anchor, float*
     return TTF_OK;
 }
 
-// 1: clips that qualify take the single-launch pass (ttf_fused.cu); 0: the kernel sequence.  Off unless
-// TTF_SINGLE_LAUNCH=1 is in the environment or ttf_set_single_launch(1) was called: on the clips measured so far
-// the kernel sequence spread over streams is the faster of the two.
-static int g_use_fused = -1;
-static bool use_fused(const Problem& p, const void* out_tokens) {
-    if (g_use_fused < 0) {
-        const char* e = getenv("TTF_SINGLE_LAUNCH");
-        g_use_fused = (e && e[0] == '1') ? 1 : 0;
-    }
-    return g_use_fused == 1 && fused_eligible(p) && reinterpret_cast<uintptr_t>(out_tokens) % 16 == 0;
-}
-
 static int compress_impl(const Problem& p, void* ws, void* out_tokens, int* out_count, int* out_pos,
                          cudaStream_t st) {
     Scratch s;
     carve_scratch(p, ws, &s);
-    if (use_fused(p, out_tokens)) {
-        cudaError_t e;
-        { ProfScope ps(st, PK_FUSED);
-          e = launch_fused(p, s, nullptr, s.shat, s.dst, s.keep, s.fuse_cnt, out_tokens, out_pos, out_count, st); }
-        return e == cudaSuccess ? TTF_OK : cuda_fail(e);
-    }
     int rc = run_front(p, s, nullptr, s.shat, s.dst, s.keep, st);
     if (rc != TTF_OK) return rc;
     cudaError_t e;
@@ -208,12 +243,6 @@ static int query_impl(const Problem& p, void* ws, int* out_anchor, unsigned char
     float* shat = out_sim ? out_sim : s.shat;
     int* dst = out_dst ? out_dst : s.dst;
     unsigned char* keep = out_keep ? out_keep : s.keep;
-    if (use_fused(p, nullptr)) {
-        cudaError_t e;
-        { ProfScope ps(st, PK_FUSED);
-          e = launch_fused(p, s, out_anchor, shat, dst, keep, out_fuse, nullptr, nullptr, nullptr, st); }
-        return e == cudaSuccess ? TTF_OK : cuda_fail(e);
-    }
     int rc = run_front(p, s, out_anchor, shat, dst, keep, st);
     if (rc != TTF_OK) return rc;
     if (out_fuse) {
@@ -281,12 +310,64 @@ const char* ttf_status_string(int status) {
         case TTF_ERR_UNSUPPORTED: return "TTF_ERR_UNSUPPORTED";
         case TTF_ERR_WORKSPACE: return "TTF_ERR_WORKSPACE";
         case TTF_ERR_CUDA: return "TTF_ERR_CUDA";
+        case TTF_ERR_TIMEOUT: return "TTF_ERR_TIMEOUT";
         case TTF_ERR_STATIC_LIMIT: return "TTF_ERR_STATIC_LIMIT";
         default: return "TTF_ERR_UNKNOWN";
     }
 }
 
 int ttf_last_cuda_error(void) { return tl_cuda_error; }
+
+static int read_status_words(const std::vector<const int*>& words, int* host_status) {
+    *host_status = TTF_OK;
+    for (const int* hdr : words) {
+        int v = 0;
+        cudaError_t e = cudaMemcpy(&v, hdr + HDR_ERROR, sizeof(int), cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (v) *host_status = TTF_ERR_TIMEOUT;
+    }
+    return TTF_OK;
+}
+
+int ttf_last_device_status(ttf_stream_t stream, int* host_status) {
+    if (!host_status) return TTF_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    int dev = 0;
+    e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    std::vector<const int*> words;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_scratch.find(std::make_pair(dev, st));
+        if (it != g_scratch.end()) words = it->second.status_words;
+    }
+    return read_status_words(words, host_status);     // no call of the library on this stream yet: TTF_OK
+}
+
+int ttf_workspace_status(const void* workspace, ttf_stream_t stream, int* host_status) {
+    if (!host_status) return TTF_ERR_INVALID_ARG;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
+    if (e != cudaSuccess) return cuda_fail(e);
+    void* ws = const_cast<void*>(workspace);
+    if (!ws) {                                   // NULL: the built-in array of ttf_query_static
+        int rc = static_scratch_address(&ws);
+        if (rc != TTF_OK) return rc;
+    }
+    return read_status_words(std::vector<const int*>(1, reinterpret_cast<const int*>(ws)), host_status);
+}
+
+int ttf_debug_set_wait(int poll_limit, int tx_extra_bytes) {
+    if (poll_limit < 1 || tx_extra_bytes < 0 || tx_extra_bytes % 16 != 0 || tx_extra_bytes > 1024) return TTF_ERR_INVALID_ARG;
+    g_wait_limit.store(poll_limit);
+    g_wait_tx_extra.store(tx_extra_bytes);
+    return TTF_OK;
+}
+
+int ttf_debug_func_attr_needed(const void* key, int device, size_t bytes) {
+    return g_func_attr.needs(key, device, bytes) ? 1 : 0;
+}
 
 int ttf_workspace_bytes(int F, int H, int W, int C, int r, int dtype, size_t* bytes) {
     if (!bytes) return TTF_ERR_INVALID_ARG;
@@ -460,7 +541,9 @@ static int batch_on_streams(const void* const* features, int nclips, int F, int 
     BatchLanes* L = nullptr;
     int rc = batch_lanes(&L);
     if (rc != TTF_OK) return rc;
-    const int lanes = nclips < kBatchStreams ? nclips : kBatchStreams;
+    int want = g_sched_lanes.load();
+    if (want < 1 || want > kBatchStreams) want = kBatchStreams;
+    const int lanes = nclips < want ? nclips : want;
     cudaError_t e = cudaEventRecord(L->fork, st);
     for (int i = 0; i < lanes && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(L->s[i], L->fork, 0);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -468,6 +551,18 @@ static int batch_on_streams(const void* const* features, int nclips, int F, int 
     for (int n = 0; n < nclips && first_rc == TTF_OK; ++n)
         first_rc = ttf_compress(features[n], F, H, W, C, r, t, dtype, out_tokens[n], out_count[n], out_pos_thw[n],
                                 (ttf_stream_t)L->s[n % lanes]);
+    {   // the caller asks about the batch through its own stream: point it at the lanes' error words
+        int dev = 0;
+        std::vector<const int*> words;
+        if (cudaGetDevice(&dev) == cudaSuccess) {
+            std::lock_guard<std::mutex> lk(g_mu);
+            for (int i = 0; i < lanes; ++i) {
+                auto it = g_scratch.find(std::make_pair(dev, L->s[i]));
+                if (it != g_scratch.end()) words.insert(words.end(), it->second.status_words.begin(), it->second.status_words.end());
+            }
+            g_scratch[std::make_pair(dev, st)].status_words = words;
+        }
+    }
     // always join, also after a failed launch, so that the caller's stream (or capture) is whole again
     for (int i = 0; i < lanes; ++i) {
         cudaError_t e2 = cudaEventRecord(L->join[i], L->s[i]);
@@ -478,10 +573,19 @@ static int batch_on_streams(const void* const* features, int nclips, int F, int 
     return e == cudaSuccess ? TTF_OK : cuda_fail(e);
 }
 
-int ttf_set_single_launch(int on) {
-    const int before = g_use_fused == 1 ? 1 : 0;
-    g_use_fused = on ? 1 : 0;
-    return before;
+int ttf_set_match_kernel(int which) {
+    if (which < 0 || which > 2) return TTF_ERR_INVALID_ARG;
+    g_match_kernel.store(which);
+    return TTF_OK;
+}
+
+int ttf_set_schedule(int clips_in_flight, int l2_mode, int resident_pct) {
+    if (clips_in_flight < 0 || clips_in_flight > kBatchStreams || l2_mode < 0 || l2_mode > 2 || resident_pct < 0 ||
+        resident_pct > 100) return TTF_ERR_INVALID_ARG;
+    g_sched_lanes.store(clips_in_flight);
+    g_sched_l2_mode.store(l2_mode);
+    g_sched_res_pct.store(resident_pct);
+    return TTF_OK;
 }
 
 int ttf_compress_batch(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
@@ -494,27 +598,7 @@ int ttf_compress_batch(const void* const* features, int nclips, int F, int H, in
     Problem p;
     int rc = make_problem(features[0], F, H, W, C, r, t, dtype, &p);
     if (rc != TTF_OK) return rc;
-    bool batched = nclips > 1 && use_fused(p, out_tokens[0]) && !g_prof_on;
-    for (int n = 1; n < nclips && batched; ++n)
-        batched = reinterpret_cast<uintptr_t>(features[n]) % 16 == 0 && reinterpret_cast<uintptr_t>(out_tokens[n]) % 16 == 0;
-    Scratch s;
-    carve_scratch(p, nullptr, &s);
-    const size_t stride = s.bytes;
-    const int chunk = nclips < kFusedBatchMax ? nclips : kFusedBatchMax;
-    if (!batched) return batch_on_streams(features, nclips, F, H, W, C, r, t, dtype, out_tokens, out_count, out_pos_thw, st);
-    void* ws = nullptr;
-    rc = cached_scratch(stride * chunk, st, &ws);
-    if (rc != TTF_OK) return rc;
-    rc = clear_control_blocks(ws, stride, chunk, st);
-    if (rc != TTF_OK) return rc;
-    carve_scratch(p, ws, &s);
-    for (int base = 0; base < nclips; base += kFusedBatchMax) {
-        const int m = nclips - base < kFusedBatchMax ? nclips - base : kFusedBatchMax;
-        cudaError_t e = launch_fused_batch(p, s, (long long)stride, m, features + base, out_tokens + base,
-                                           out_pos_thw + base, out_count + base, st);
-        if (e != cudaSuccess) return cuda_fail(e);
-    }
-    return TTF_OK;
+    return batch_on_streams(features, nclips, F, H, W, C, r, t, dtype, out_tokens, out_count, out_pos_thw, st);
 }
 
 int ttf_compress_segment(const void* features, int F, int H, int W, int C, int r, float t, int dtype,

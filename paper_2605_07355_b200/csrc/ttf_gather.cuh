@@ -1,5 +1,5 @@
 // Rank/select helpers of the output-driven gather and the fuse-count bookkeeping, shared by the stand-alone
-// compaction kernels and the fused single-launch pass.
+// compaction kernels.
 #pragma once
 
 #include "ttf_internal.cuh"
@@ -11,15 +11,15 @@ constexpr int kScanChunks = 4;       // frame counts per lane fetched at once by
 
 // Tokens fused into each anchor cell j: |{(k,i): k != a, keep = 0, dst = j}|, gather-side (every cell looks at
 // the (2r+1)^2 x (F-1) tokens that can point to it), integer, order-free.  Run by whole CTAs: block `b` of `nb`,
-// one warp per cell.  The lanes split the (frame, window cell) pairs of the cell and fetch both flags of four
+// one warp per cell (any number of warps per CTA).  The lanes split the (frame, window cell) pairs of the cell and fetch both flags of four
 // pairs at a time without testing one before loading the other, so the loads of a lane overlap instead of
 // forming a chain of dependent round trips.
 __device__ __forceinline__ void fuse_count_cta(int F, int H, int W, int r, int a, const unsigned char* keep,
                                                const int* dst, int* fuse_cnt, int b, int nb) {
     if (fuse_cnt == nullptr) return;
     const int N = H * W;
-    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-    for (int j = b * kCopyWarps + w; j < N; j += nb * kCopyWarps) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, warps = blockDim.x >> 5;
+    for (int j = b * warps + w; j < N; j += nb * warps) {
         const int y = j / W, x = j - y * W;
         const int y_lo = max(0, y - r), x_lo = max(0, x - r);
         const int nx = min(W - 1, x + r) - x_lo + 1, wsz = (min(H - 1, y + r) - y_lo + 1) * nx;

@@ -13,13 +13,12 @@ constexpr int kWarpPrefixMaxF = 1024;  // frame counts up to this are scanned by
 constexpr int kHdrInts = 64;
 constexpr int kStatReplicas = 16;      // copies of the frame statistics, so that the CTAs that read them at the
                                        // same moment do not all queue on the same few cache lines
-constexpr int kFusedMaxSplit = 4;     // fused pass: at most this many token ranges per frame in the sweep
-constexpr int kResolveMaxF = 256;      // single-launch pass: clips up to this many frames (every CTA takes the arg max itself)
 
 // header words of the scratch block
-enum { HDR_ANCHOR = 0, HDR_DONE_ALL = 1, HDR_ERROR = 2,     // HDR_ERROR: a bounded wait gave up
-       HDR_BAR = 3, HDR_SWEEP = 5, HDR_EXIT = 6 };           // fused pass: barrier arrivals of the (two) CTA groups, CTAs
-                                                             // that completed a sweep, CTAs done; zero between calls
+enum { HDR_ANCHOR = 0,          // anchor frame a*
+       HDR_DONE_ALL = 1,        // arrival counter of the statistics CTAs (zero between calls)
+       HDR_ERROR = 2,           // a bounded wait of this call gave up (cleared by the first kernel of every call)
+       HDR_GATHER_DONE = 3 };   // arrival counter of the gather's warps (zero between calls)
 
 // Problem description handed to every launcher.
 struct Problem {
@@ -38,6 +37,10 @@ struct Problem {
     int anchor_arg;     // explicit anchor frame
     int emit_anchor;    // 1: X' starts with the N anchor rows (Eq. xprime_stack); 0: streaming segment, sources only
     int pos_t_offset;   // added to the frame coordinate of every emitted position
+    int l2_mode;        // L2 eviction priorities of the passes over X: 0 none; 1: frames < res_frames default priority,
+                        // everything else evict-first; 2: frames < res_frames evict-last, everything else evict-first
+    int res_frames;     // leading frames of the clip that the sweep asks L2 to keep for the matching pass
+    int use_tc;         // 1: the matching step runs on tcgen05 (ttf_match_tc.cu), norms from the sweep
 };
 
 // Device pointers carved out of one scratch allocation.
@@ -45,7 +48,7 @@ struct Scratch {
     int* hdr;           // [kHdrInts]  anchor frame, arrival counter of the anchor-pick slices
     int* cnt;           // [F]   preserved tokens per source frame (Eq. gating summed over a frame)
     int* prefix;        // [F+1] exclusive scan of cnt, only used when F > kWarpPrefixMaxF
-    float* S;           // [F, C] per-frame channel sums ([kFusedMaxSplit, F, C] token-range parts in the fused pass)
+    float* S;           // [F, C] per-frame channel sums
     float* Dp;          // [kStatReplicas][nsl, F] per-slice share of <S_k, g>
     float* Qp;          // [kStatReplicas][nsl, F] per-slice share of |S_k|^2
     float* Gp;          // [kStatReplicas][nsl]    per-slice share of |g|^2
@@ -54,6 +57,9 @@ struct Scratch {
     int* dst;           // [F*N] best anchor cell (Eq. dst)
     unsigned char* keep;// [F*N] retention mask (Eq. mask)
     int* fuse_cnt;      // [N]   tokens fused into each anchor cell
+    float* tc_part;     // tcgen05 matching: partial window sums [tile][piece][(2r+1)^2][128] (pieces > 1 only)
+    int* tc_cnt;        // tcgen05 matching: arrival counter per tile (zero between calls)
+    int tc_tiles;       // number of those counters
     size_t bytes;       // total, multiple of 256
 };
 
@@ -78,7 +84,15 @@ inline bool uses_mma_match(const Problem& p) {
 }
 
 // The sweep stores per-token partial squared norms only for the kernels that read them.
-inline bool needs_sweep_norms(const Problem& p) { return !uses_mma_match(p) || p.r == 2; }
+inline bool needs_sweep_norms(const Problem& p) { return !uses_mma_match(p) || p.r == 2 || p.use_tc; }
+
+// tcgen05 matching (ttf_match_tc.cu)
+bool tc_match_eligible(const Problem& p);
+int tc_match_pieces(const Problem& p);
+size_t tc_match_part_floats(const Problem& p);
+size_t tc_match_tiles(const Problem& p);
+cudaError_t launch_match_tc(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
+                            unsigned char* keep, cudaStream_t st);
 
 // Fills the offsets (base may be NULL to only compute `bytes`).
 void carve_scratch(const Problem& p, void* base, Scratch* s);
@@ -102,20 +116,16 @@ cudaError_t launch_sim_histogram(const float* sim, const int* anchor, int F, int
 // Optional mean fusion (ttf_fuse.cu; not the paper's method): overwrites the anchor block of out_tokens.
 cudaError_t launch_fuse_mean(const Problem& p, const Scratch& s, void* out_tokens, cudaStream_t st);
 
-// The whole pass in one cooperative launch (ttf_fused.cu).  out_tokens == NULL stops before the compaction.
-bool fused_eligible(const Problem& p);
-int fused_grid();                       // CTAs of the fused kernel on the current device
-void set_fused_ctas_per_sm(int n);      // 1 or 2
-cudaError_t launch_fused(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
-                         unsigned char* keep, int* fuse_cnt, void* out_tokens, int* out_pos, int* out_count,
-                         cudaStream_t st);
-
-constexpr int kFusedBatchMax = 32;      // clips per launch of the batched pass
-cudaError_t launch_fused_batch(const Problem& p, const Scratch& s, long long ws_stride, int nclips,
-                               const void* const* X, void* const* out_tokens, int* const* out_pos,
-                               int* const* out_count, cudaStream_t st);
-
 int sm_count();   // SMs of the current device (cached per device)
+
+// cudaFuncAttributeMaxDynamicSharedMemorySize belongs to a function in the context of ONE device: set it the first
+// time `func` is launched on the current device (and again if a larger size is asked for).
+cudaError_t ensure_dynamic_smem(const void* func, size_t bytes);
+
+// Bounded waits: polls of an mbarrier before a waiter gives up, and extra bytes announced to it (always 0 outside
+// the test that makes a wait run out; see ttf_debug_set_wait).
+int wait_poll_limit();
+int wait_tx_extra();
 
 inline AnchorSrc make_anchor_src(const Problem& p, const Scratch& s, int* out_anchor) {
     AnchorSrc a;
@@ -181,6 +191,21 @@ __device__ __forceinline__ void trace_mark(int* hdr, int id, bool end) {
 __device__ __forceinline__ void trace_mark(int*, int, bool) {}
 #endif
 
+// L2 eviction-priority policies (createpolicy) and 16-byte loads that carry one
+__device__ __forceinline__ uint64_t l2_policy(int kind) {     // 0 evict_first, 1 evict_normal, 2 evict_last
+    uint64_t p;
+    if (kind == 0) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    else if (kind == 2) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint4 ldcg_hint16(const void* p, uint64_t pol) {
+    uint4 v;
+    asm volatile("ld.global.cg.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
+    return v;
+}
+
 struct bf16_t { uint16_t bits; };   // storage type only: all arithmetic is on the widened fp32 value
 
 __device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
@@ -193,6 +218,10 @@ template <> struct Loader<float, 4> {
     using Raw = float4;
     static __device__ __forceinline__ Raw load_raw(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
     static __device__ __forceinline__ Raw load_raw_cg(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+    static __device__ __forceinline__ Raw load_raw_hint(const float* p, uint64_t pol) {
+        const uint4 v = ldcg_hint16(p, pol);
+        return make_float4(__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w));
+    }
     static __device__ __forceinline__ Raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[4]) { x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
     static __device__ __forceinline__ void load(const float* p, float (&x)[4]) { unpack(load_raw(p), x); }
@@ -201,6 +230,7 @@ template <> struct Loader<float, 1> {
     using Raw = float;
     static __device__ __forceinline__ Raw load_raw(const float* p) { return __ldg(p); }
     static __device__ __forceinline__ Raw load_raw_cg(const float* p) { return __ldcg(p); }
+    static __device__ __forceinline__ Raw load_raw_hint(const float* p, uint64_t) { return __ldcg(p); }
     static __device__ __forceinline__ Raw zero() { return 0.f; }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[1]) { x[0] = v; }
     static __device__ __forceinline__ void load(const float* p, float (&x)[1]) { x[0] = __ldg(p); }
@@ -209,6 +239,7 @@ template <> struct Loader<bf16_t, 8> {
     using Raw = uint4;
     static __device__ __forceinline__ Raw load_raw(const bf16_t* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
     static __device__ __forceinline__ Raw load_raw_cg(const bf16_t* p) { return __ldcg(reinterpret_cast<const uint4*>(p)); }
+    static __device__ __forceinline__ Raw load_raw_hint(const bf16_t* p, uint64_t pol) { return ldcg_hint16(p, pol); }
     static __device__ __forceinline__ Raw zero() { return make_uint4(0, 0, 0, 0); }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[8]) {
         x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);
@@ -224,6 +255,7 @@ template <> struct Loader<bf16_t, 1> {
     static __device__ __forceinline__ Raw load_raw_cg(const bf16_t* p) {
         return __uint_as_float(static_cast<uint32_t>(__ldcg(reinterpret_cast<const unsigned short*>(p))) << 16);
     }
+    static __device__ __forceinline__ Raw load_raw_hint(const bf16_t* p, uint64_t) { return load_raw_cg(p); }
     static __device__ __forceinline__ Raw zero() { return 0.f; }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[1]) { x[0] = v; }
     static __device__ __forceinline__ void load(const bf16_t* p, float (&x)[1]) { x[0] = load_raw(p); }

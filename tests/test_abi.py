@@ -87,11 +87,11 @@ def test_batch_and_variant_entry_points_validate_before_any_cuda_call(lib):
     assert h(arr, 2, 4, 4, 4, 8, -1, 0.7, 0, arr, ctypes.cast(counts, ctypes.c_void_p), arr) == 1
     assert lib.ttf_compress_mean(None, 4, 4, 4, 8, 1, 0.7, 0, fake, fake, fake, None) == 1
     assert lib.ttf_compress_mean(fake, 4, 4, 4, 8, 1, 0.7, 2, fake, fake, fake, None) == 1
-    ms = (ctypes.c_double * 6)()
-    assert lib.ttf_profile_stages(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, 0, ms, 6, None) == 1   # reps < 1
-    assert lib.ttf_profile_stages(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, 1, None, 6, None) == 1
-    before = lib.ttf_set_single_launch(1)
-    assert lib.ttf_set_single_launch(before) == 1 and lib.ttf_set_single_launch(before) == before
+    ms = (ctypes.c_double * 5)()
+    assert lib.ttf_profile_stages(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, 0, ms, 5, None) == 1   # reps < 1
+    assert lib.ttf_profile_stages(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, 1, None, 5, None) == 1
+    assert lib.ttf_set_schedule(9, 0, 0) == 1 and lib.ttf_set_schedule(0, 3, 0) == 1 and lib.ttf_set_schedule(0, 0, 101) == 1
+    assert lib.ttf_set_schedule(0, 0, 0) == 0
 
 
 def test_decode_alignment_helper():
@@ -110,3 +110,28 @@ def test_flop_counter_reproduces_table3():
     assert A.window_pairs(16, 16, 1) == 2116 and A.window_pairs(32, 32, 2) == 23716
     assert A.matching_flops(32, 16, 16, 1152, 1) < A.matching_flops_nominal(32, 256, 1152, 1)
     assert A.pass_bytes(32, 256, 4096, 2, 2703) == 32 * 256 * 4096 * 2 + 2703 * 8192 + 2703 * 12 + 4
+
+
+def test_dynamic_shared_memory_limits_are_recorded_per_function_and_device(lib):
+    """a function attribute set in one device's context says nothing about another device"""
+    import ctypes
+    need = lib.ttf_debug_func_attr_needed
+    need.restype = ctypes.c_int
+    need.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t]
+    key_a, key_b = ctypes.c_void_p(0x1000), ctypes.c_void_p(0x2000)
+    assert need(key_a, 0, 65536) == 1            # first launch of a on device 0: set it
+    assert need(key_a, 0, 65536) == 0            # already set there
+    assert need(key_a, 1, 65536) == 1            # device 1 has its own context
+    assert need(key_b, 0, 65536) == 1            # another function
+    assert need(key_a, 0, 32768) == 0            # a smaller request is covered
+    assert need(key_a, 0, 131072) == 1           # a larger one is not
+    assert need(key_a, 1, 65536) == 0
+
+
+def test_status_entry_points_validate(lib):
+    import ctypes
+    assert lib.ttf_last_device_status(None, None) == 1
+    assert lib.ttf_workspace_status(None, None, None) == 1
+    assert lib.ttf_debug_set_wait(0, 0) == 1 and lib.ttf_debug_set_wait(8, 8) == 1 and lib.ttf_debug_set_wait(8, 2048) == 1
+    assert lib.ttf_debug_set_wait(1 << 18, 0) == 0
+    assert lib.ttf_status_string(5) == b"TTF_ERR_TIMEOUT" and lib.ttf_status_string(6) == b"TTF_ERR_STATIC_LIMIT"

@@ -1,4 +1,4 @@
-"""GPU parity of the batch entry point and of the single-launch variant of the pass (through the C ABI)."""
+"""GPU parity of the batch entry points (through the C ABI)."""
 import numpy as np
 import pytest
 import torch
@@ -21,13 +21,6 @@ def assert_same_as_single(Xs, r, t, outs):
         L = int(a[1].item())
         assert int(cnts[j].item()) == L, (j, int(cnts[j].item()), L)
         assert torch.equal(toks[j][:L], a[0][:L]) and torch.equal(poss[j][:L], a[2][:L]), j
-
-
-@pytest.fixture
-def single_launch():
-    before = P.ttf_set_single_launch(True)
-    yield
-    P.ttf_set_single_launch(before)
 
 
 def test_batch_on_library_streams_matches_single_calls_and_oracle():
@@ -61,47 +54,6 @@ def test_batch_small_and_fp32_and_stream_order():
     assert_same_as_single(Xs[:1], 1, 0.7, one)
     with pytest.raises(ValueError):
         P.ttf_compress_batch([Xs[0], Xs[1][:2]], 1, 0.7)
-
-
-SHAPES = [(1, 4, 4, 32, 1), (2, 3, 5, 40, 1), (6, 5, 6, 264, 0), (17, 3, 3, 72, 1), (33, 2, 3, 8, 1),
-          (9, 4, 6, 1032, 1), (40, 7, 9, 512, 1)]
-
-
-@pytest.mark.parametrize("shape", SHAPES)
-def test_single_launch_small_shapes(single_launch, shape):
-    F, H, W, C, r = shape
-    X = corr_clip(F, H, W, C, seed=sum(shape), dtype="bf16")
-    for t in (0.7, 0.5):
-        check_clip(X, r, t)
-
-
-def test_single_launch_paper_shaped_and_fixed_anchors(single_launch):
-    s = clips.CONFIGS["vl2b_cal"]
-    rep = check_clip(clips.make_clip(s), s.r, s.t)
-    assert abs(rep["rho"] - 0.67) < 0.02
-    X = corr_clip(5, 6, 7, 256, seed=5, dtype="bf16")
-    for mode, frame in ((1, 0), (2, 0), (3, 2)):
-        rep = check_clip(X, 1, 0.7, anchor_mode=mode, anchor_frame=frame)
-        assert rep["anchor"] == {1: 0, 2: 4, 3: 2}[mode]
-    check_clip(np.zeros((3, 3, 3, 16), np.uint16), 1, 0.5)           # all-zero bf16 clip
-
-
-def test_single_launch_batch_two_groups():
-    s = clips.CONFIGS["vl2b_cal"]
-    Xs = [to_device(clips.make_clip(s, s.seed + j)) for j in range(5)]      # odd count: the groups end unevenly
-    ref = [P.ttf_compress(x, s.r, s.t) for x in Xs]
-    torch.cuda.synchronize()
-    before = P.ttf_set_single_launch(True)
-    try:
-        for rep in range(2):                     # twice: the control words must be back at zero after a launch
-            toks, cnts, poss = P.ttf_compress_batch(Xs, s.r, s.t)
-            torch.cuda.synchronize()
-            for j in range(len(Xs)):
-                L = int(ref[j][1].item())
-                assert int(cnts[j].item()) == L
-                assert torch.equal(toks[j][:L], ref[j][0][:L]) and torch.equal(poss[j][:L], ref[j][2][:L])
-    finally:
-        P.ttf_set_single_launch(before)
 
 
 def test_host_batch_matches_device_calls():
@@ -143,23 +95,6 @@ def test_bench_configuration_full_size_against_oracle():
         assert (to_bits(toks[j][:L]) == forced.tokens).all()
         rhos.append(1.0 - L / s.tokens)
     assert abs(float(np.mean(rhos)) - 0.67) < 0.03
-
-
-def test_single_launch_batch_longer_than_one_launch():
-    """more clips than one cooperative launch takes (32): the batch is cut into launches that reuse the scratch"""
-    Xs = [to_device(corr_clip(3, 4, 4, 64, seed=100 + j, dtype="bf16")) for j in range(35)]
-    ref = [P.ttf_compress(x, 1, 0.7) for x in Xs]
-    torch.cuda.synchronize()
-    before = P.ttf_set_single_launch(True)
-    try:
-        toks, cnts, poss = P.ttf_compress_batch(Xs, 1, 0.7)
-        torch.cuda.synchronize()
-    finally:
-        P.ttf_set_single_launch(before)
-    for j in range(len(Xs)):
-        L = int(ref[j][1].item())
-        assert int(cnts[j].item()) == L
-        assert torch.equal(toks[j][:L], ref[j][0][:L]) and torch.equal(poss[j][:L], ref[j][2][:L])
 
 
 def test_host_batch_fp32_and_single_clip():
@@ -212,11 +147,7 @@ def test_multi_block_scratch_after_another_shape_on_the_same_stream():
     torch.cuda.synchronize()
     with torch.cuda.stream(st):
         P.ttf_compress(big, 1, 0.7, stream=st)                     # fills the stream's scratch with its arrays
-        before = P.ttf_set_single_launch(True)
-        try:
-            toks, cnts, poss = P.ttf_compress_batch(small, 1, 0.7, stream=st)
-        finally:
-            P.ttf_set_single_launch(before)
+        toks, cnts, poss = P.ttf_compress_batch(small, 1, 0.7, stream=st)
     st.synchronize()
     for j in range(len(small)):
         L = int(ref[j][1].item())
