@@ -59,6 +59,20 @@ typedef enum {
  * or an explicit frame (e.g. the rolling anchor of a streaming segment, Sec. 5 D3) */
 typedef enum { TTF_ANCHOR_AUTO = 0, TTF_ANCHOR_FIRST = 1, TTF_ANCHOR_LAST = 2, TTF_ANCHOR_EXPLICIT = 3 } ttf_anchor_mode;
 
+/* order of the compressed sequence: the paper's (anchor-frame rows precede the preserved source rows, Eq.
+ * xprime_stack), or every retained token in ascending flat index k*N + i (the anchor rows where they fall) */
+typedef enum { TTF_ORDER_ANCHOR_FIRST = 0, TTF_ORDER_NATURAL = 1 } ttf_order;
+
+/* Options of the _ex entry points; a NULL pointer means all zero: the automatic anchor, the paper's order, raw
+ * (k, y, x) positions. */
+typedef struct {
+    int anchor_mode;   /* a ttf_anchor_mode                                                                      */
+    int anchor_frame;  /* the frame of TTF_ANCHOR_EXPLICIT, in [0, F); ignored otherwise                         */
+    int order;         /* a ttf_order                                                                            */
+    int pos_base;      /* >= 0, added to all three coordinates of every emitted position (e.g. the index of the  */
+                       /* first visual token in the prompt, as multimodal rotary embeddings count it)            */
+} ttf_options;
+
 typedef struct CUstream_st* ttf_stream_t;      /* same type as cudaStream_t */
 
 /* Human-readable name of a ttf_status. Never NULL. */
@@ -120,11 +134,12 @@ int ttf_compress(const void* features, int F, int H, int W, int C, int r, float 
  * A batch of clips of one shape in one call (the long-video workload: the clips of a request processed
  * concurrently; Sec. 3 treats every clip independently, so this is scheduling only and each clip's results are
  * exactly those of ttf_compress).  features, out_tokens, out_count and out_pos_thw are HOST arrays of nclips
- * DEVICE pointers, read before the call returns.  The clips are spread round-robin over eight streams that the
- * library keeps per device; these fork from `stream` and join it again through events, so the call is
+ * DEVICE pointers, read before the call returns.  The clips are spread round-robin over up to eight streams ("lanes")
+ * that the library keeps per device; these fork from `stream` and join it again through events, so the call is
  * asynchronous, ordered on `stream` like any other, and can be captured in a CUDA graph.  The kernels of one clip
- * leave much of the GPU idle while they ramp up and drain; with several clips in flight those gaps are filled.
- * Scratch: one block per internal stream, from the cache.  The streams, their events and the scratch are created by
+ * leave much of the GPU idle while they ramp up and drain; with several clips in flight those gaps are filled
+ * (ttf_set_schedule sets the number of lanes).  Within a lane the clips form a chain on two scratch blocks used in
+ * turn: the sweep of a clip runs beside the gather of the clip before it.  The streams, their events and the scratch are created by
  * the first call on a device: make that call outside any stream capture.
  */
 int ttf_compress_batch(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
@@ -141,16 +156,13 @@ int ttf_compress_batch(const void* const* features, int nclips, int F, int H, in
 int ttf_set_match_kernel(int which);
 
 /*
- * Schedule of ttf_compress_batch and L2 use of the passes over X (the paper has no counterpart).  Eq. (auto_anchor)
- * needs all of X before any token can be matched, so X is read twice; the second read is free only for what is still
- * in L2.  clips_in_flight (0 = automatic, at most 8) bounds how many clips of a batch run concurrently.  l2_mode
- * selects the L2 eviction priorities the kernels attach to their accesses to X: 0 none; 1 the first
- * ceil(F * resident_pct / 100) frames of a clip are read with the default priority by the sweep and every other
- * access (the remaining frames, the matching pass's source rows, the gather's rows and its output) as evict-first;
- * 2 the same with evict-last for the leading frames.  Results do not depend on any of this.  Process-wide; takes
- * effect with the next call.
+ * Schedule of ttf_compress_batch (the paper has no counterpart).  clips_in_flight bounds how many clips of a batch run
+ * concurrently (lanes): 0 = automatic, else 1 to 8.  Eq. (auto_anchor) needs all of X before any token can be matched,
+ * so X is read twice; with few clips in flight the second read finds the clip in L2 but the kernels of one clip leave
+ * much of the GPU idle while they ramp up and drain, with many the gaps are filled but the clips displace one another
+ * in L2.  Results do not depend on it.  Process-wide; takes effect with the next call.
  */
-int ttf_set_schedule(int clips_in_flight, int l2_mode, int resident_pct);
+int ttf_set_schedule(int clips_in_flight);
 
 /* Same, with caller-owned scratch: `workspace` must be 256-byte aligned device memory of at least
  * ttf_workspace_bytes(...) bytes that no other in-flight call uses.  Allocates nothing. */
@@ -177,18 +189,23 @@ int ttf_query_ws(const void* features, int F, int H, int W, int C, int r, float 
                  int* out_fuse_cnt, void* workspace, size_t workspace_bytes, ttf_stream_t stream);
 
 /*
- * ttf_compress / ttf_query with the anchor rule chosen by the caller (Table 1 rows "first", "last", "auto";
- * ablation A2).  anchor_mode is a ttf_anchor_mode; anchor_frame is used only by TTF_ANCHOR_EXPLICIT and must
- * lie in [0, F).  With a fixed anchor the frame-mean cosines of Eq. (auto_anchor) are not evaluated.
- * Everything else is as in ttf_compress / ttf_query (scratch from the per-stream cache).
+ * ttf_compress / ttf_query / ttf_compress_batch with options (Table 1 rows "first", "last", "auto" and ablation A2 for
+ * the anchor rule; Eqs. xprime_stack and compress_pos for order and positions).  With a fixed anchor the frame-mean
+ * cosines of Eq. (auto_anchor) are not evaluated.  In natural order row j of out_tokens is the j-th retained token in
+ * ascending flat index, anchor rows included (the two orders coincide when the anchor is frame 0).  Positions are
+ * (pos_base + k, pos_base + y, pos_base + x).  The query outputs do not depend on order or pos_base.  Everything
+ * else is as in the plain entry points (scratch from the per-stream cache).
  */
 int ttf_compress_ex(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
-                    int anchor_mode, int anchor_frame,
+                    const ttf_options* options,
                     void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream);
 int ttf_query_ex(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
-                 int anchor_mode, int anchor_frame,
+                 const ttf_options* options,
                  int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
                  int* out_fuse_cnt, ttf_stream_t stream);
+int ttf_compress_batch_ex(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
+                          int dtype, const ttf_options* options,
+                          void* const* out_tokens, int* const* out_count, int* const* out_pos_thw, ttf_stream_t stream);
 
 /*
  * ttf_compress with MEAN fusion.  This is NOT the paper's method: Sec. 3 (Threshold Gating) replaces a fused token

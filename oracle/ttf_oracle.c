@@ -198,20 +198,26 @@ void ttf_oracle_fuse_count(const uint8_t* keep, const int* dst, int F, int N, in
  * P = {(k, y_i, x_i)} with m_{k,i} = 1, anchor rows first, then source rows by ascending flat index.
  * Rows are copied byte for byte (row_bytes = C * element size).  index_out[j] = flat index of output row j.
  * Returns L' = N + P (Eq. Lpre).  Any of out_tokens / out_pos / index_out may be NULL.
+ * natural != 0 gives the other reading of "ordered index set": one pass in ascending flat index, the anchor rows
+ * where they fall.  pos_base is added to all three coordinates (the offset at which a prompt places its visual
+ * tokens).
  */
 int ttf_oracle_compact(const void* Xbytes, size_t row_bytes, const uint8_t* keep, int F, int H, int W, int a,
-                       void* out_tokens, int* out_pos, int* index_out) {
+                       int natural, int pos_base, void* out_tokens, int* out_pos, int* index_out) {
     const int N = H * W;
     int L = 0;
-    for (int pass = 0; pass < 2; ++pass) {
+    for (int pass = natural ? 1 : 0; pass < 2; ++pass) {
         for (int k = 0; k < F; ++k) {
-            if ((pass == 0) != (k == a)) continue;      /* pass 0: the anchor frame; pass 1: source frames */
+            /* paper's order: pass 0 = the anchor frame, pass 1 = the source frames; natural: one pass over all */
+            if (!natural && (pass == 0) != (k == a)) continue;
             for (int i = 0; i < N; ++i) {
                 size_t f = (size_t)k * N + i;
                 if (!keep[f]) continue;
                 if (out_tokens)
                     memcpy((char*)out_tokens + (size_t)L * row_bytes, (const char*)Xbytes + f * row_bytes, row_bytes);
-                if (out_pos) { out_pos[3 * L + 0] = k; out_pos[3 * L + 1] = i / W; out_pos[3 * L + 2] = i % W; }
+                if (out_pos) {
+                    out_pos[3 * L + 0] = pos_base + k; out_pos[3 * L + 1] = pos_base + i / W; out_pos[3 * L + 2] = pos_base + i % W;
+                }
                 if (index_out) index_out[L] = (int)f;
                 ++L;
             }

@@ -46,7 +46,7 @@ def _load():
         lib.ttf_oracle_fuse_count.restype = None
         lib.ttf_oracle_fuse_count.argtypes = [vp, vp, c_int, c_int, c_int, vp]
         lib.ttf_oracle_compact.restype = c_int
-        lib.ttf_oracle_compact.argtypes = [vp, c_sz, vp, c_int, c_int, c_int, c_int, vp, vp, vp]
+        lib.ttf_oracle_compact.argtypes = [vp, c_sz, vp, c_int, c_int, c_int, c_int, c_int, c_int, vp, vp, vp]
         lib.ttf_oracle_restore.restype = None
         lib.ttf_oracle_restore.argtypes = [vp, c_sz, vp, vp, c_int, c_int, c_int, vp, vp]
         lib.ttf_oracle_sim_histogram.restype = None
@@ -130,9 +130,10 @@ def fuse_count(keep: np.ndarray, dst: np.ndarray, F: int, N: int, a: int) -> np.
     return out
 
 
-def compact(X: np.ndarray, keep: np.ndarray, a: int):
+def compact(X: np.ndarray, keep: np.ndarray, a: int, natural: bool = False, pos_base: int = 0):
     """Eqs. (xprime_stack), (compress_pos): returns (tokens[L', C] same dtype as X, pos[L', 3] i32,
-    index[L'] i32 flat source index of each output row, L')."""
+    index[L'] i32 flat source index of each output row, L').  natural: ascending flat index instead of the anchor
+    block first; pos_base: added to all three coordinates."""
     F, H, W, C = _shape(X)
     Xc = np.ascontiguousarray(X)
     keep = np.ascontiguousarray(keep, dtype=np.uint8)
@@ -141,7 +142,7 @@ def compact(X: np.ndarray, keep: np.ndarray, a: int):
     pos = np.empty((n, 3), dtype=np.int32)
     index = np.empty(n, dtype=np.int32)
     L = _load().ttf_oracle_compact(_ptr(Xc), C * X.dtype.itemsize, _ptr(keep), F, H, W, int(a),
-                                   _ptr(tokens), _ptr(pos), _ptr(index))
+                                   1 if natural else 0, int(pos_base), _ptr(tokens), _ptr(pos), _ptr(index))
     return tokens[:L], pos[:L], index[:L], int(L)
 
 
@@ -228,7 +229,7 @@ class OracleResult:
 
 
 def compress(X: np.ndarray, r: int, t: float, anchor_frame: Optional[int] = None,
-             forced_keep: Optional[np.ndarray] = None) -> OracleResult:
+             forced_keep: Optional[np.ndarray] = None, natural: bool = False, pos_base: int = 0) -> OracleResult:
     """The whole pass in the paper's order.  ``anchor_frame`` overrides the anchor rule (first / last /
     explicit anchors of Table 1); ``forced_keep`` replaces the gate's decisions (used after near-threshold
     differences have been accepted, so that counts, positions and rows can still be compared exactly)."""
@@ -239,5 +240,5 @@ def compress(X: np.ndarray, r: int, t: float, anchor_frame: Optional[int] = None
     s_hat, dst, second = match(X, r, a)
     keep = gate(s_hat, F, N, a, t) if forced_keep is None else np.ascontiguousarray(forced_keep, dtype=np.uint8).reshape(-1)
     fc = fuse_count(keep, dst, F, N, a)
-    tokens, pos, index, L = compact(X, keep, a)
+    tokens, pos, index, L = compact(X, keep, a, natural=natural, pos_base=pos_base)
     return OracleResult(a, cos, s_hat, dst, second, keep, fc, tokens, pos, index, L)

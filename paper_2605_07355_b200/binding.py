@@ -22,11 +22,26 @@ EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
     "ttf_query_static", "ttf_compress_ex", "ttf_query_ex", "ttf_compress_segment", "ttf_restore",
-    "ttf_sim_histogram", "ttf_compress_batch", "ttf_profile_stages", "ttf_compress_mean", "ttf_compress_host_batch",
+    "ttf_sim_histogram", "ttf_compress_batch", "ttf_compress_batch_ex", "ttf_profile_stages", "ttf_compress_mean", "ttf_compress_host_batch",
     "ttf_set_schedule", "ttf_set_match_kernel", "ttf_last_device_status", "ttf_workspace_status", "ttf_debug_set_wait", "ttf_debug_func_attr_needed",
 ]
 TTF_ERR_TIMEOUT, TTF_ERR_STATIC_LIMIT = 5, 6
 TTF_ANCHOR_AUTO, TTF_ANCHOR_FIRST, TTF_ANCHOR_LAST, TTF_ANCHOR_EXPLICIT = 0, 1, 2, 3
+TTF_ORDER_ANCHOR_FIRST, TTF_ORDER_NATURAL = 0, 1
+
+
+class TTFOptions(ctypes.Structure):
+    """ttf_options of include/ttf.h"""
+    _fields_ = [("anchor_mode", ctypes.c_int), ("anchor_frame", ctypes.c_int), ("order", ctypes.c_int),
+                ("pos_base", ctypes.c_int)]
+
+
+def _options(anchor_mode: int, anchor_frame: int, order: int, pos_base: int):
+    """NULL when everything is at its default, else a ttf_options by reference"""
+    if not (anchor_mode or anchor_frame or order or pos_base):
+        return None
+    return ctypes.byref(TTFOptions(int(anchor_mode), int(anchor_frame), int(order), int(pos_base)))
+
 TTF_STATIC_SCRATCH_BYTES = 8 << 20
 KERNEL_KINDS = ["norm_sum", "frame_stats", "match", "compact", "fuse_count"]
 
@@ -74,7 +89,7 @@ def lib() -> ctypes.CDLL:
         L.ttf_set_match_kernel.restype = i
         L.ttf_set_match_kernel.argtypes = [i]
         L.ttf_set_schedule.restype = i
-        L.ttf_set_schedule.argtypes = [i, i, i]
+        L.ttf_set_schedule.argtypes = [i]
         L.ttf_compress_mean.restype = i
         L.ttf_compress_mean.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp]
         L.ttf_compress_host_batch.restype = i
@@ -86,9 +101,11 @@ def lib() -> ctypes.CDLL:
         L.ttf_query_ws.restype = i
         L.ttf_query_ws.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp, sz, vp]
         L.ttf_compress_ex.restype = i
-        L.ttf_compress_ex.argtypes = [vp] + shape + [f, i, i, i, vp, vp, vp, vp]
+        L.ttf_compress_ex.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp]
+        L.ttf_compress_batch_ex.restype = i
+        L.ttf_compress_batch_ex.argtypes = [vp, i] + shape + [f, i, vp, vp, vp, vp, vp]
         L.ttf_query_ex.restype = i
-        L.ttf_query_ex.argtypes = [vp] + shape + [f, i, i, i, vp, vp, vp, vp, vp, vp]
+        L.ttf_query_ex.argtypes = [vp] + shape + [f, i, vp, vp, vp, vp, vp, vp, vp]
         L.ttf_compress_segment.restype = i
         L.ttf_compress_segment.argtypes = [vp] + shape + [f, i, i, vp, vp, vp, vp]
         L.ttf_restore.restype = i
@@ -150,8 +167,8 @@ def ttf_workspace_bytes(F: int, H: int, W: int, C: int, r: int, dtype: int) -> i
 def ttf_compress(features: torch.Tensor, r: int, t: float, out_tokens: Optional[torch.Tensor] = None,
                  out_count: Optional[torch.Tensor] = None, out_pos_thw: Optional[torch.Tensor] = None,
                  workspace: Optional[torch.Tensor] = None, stream=None,
-                 anchor_mode: int = 0, anchor_frame: int = 0):
-    """ttf_compress / ttf_compress_ws (ttf_compress_ex when an anchor rule other than auto is given).  Returns (out_tokens [F*H*W, C], out_count int32[1],
+                 anchor_mode: int = 0, anchor_frame: int = 0, order: int = 0, pos_base: int = 0):
+    """ttf_compress / ttf_compress_ws (ttf_compress_ex when any option is given).  Returns (out_tokens [F*H*W, C], out_count int32[1],
     out_pos_thw int32 [F*H*W, 3]); only the first out_count rows are defined.  Does not synchronise."""
     F, H, W, C = _check_features(features, "cuda")
     dev = features.device
@@ -164,11 +181,11 @@ def ttf_compress(features: torch.Tensor, r: int, t: float, out_tokens: Optional[
         out_pos_thw = torch.empty((n, 3), dtype=torch.int32, device=dev)
     with torch.cuda.device(dev):
         sp = _stream_ptr(stream)
-        if anchor_mode != 0:
+        opt = _options(anchor_mode, anchor_frame, order, pos_base)
+        if opt is not None:
             if workspace is not None:
-                raise ValueError("a fixed anchor rule uses the library's own scratch")
-            rc = lib().ttf_compress_ex(_p(features), F, H, W, C, int(r), float(t), _dtype_code(features),
-                                       int(anchor_mode), int(anchor_frame),
+                raise ValueError("the entry point with options uses the library's own scratch")
+            rc = lib().ttf_compress_ex(_p(features), F, H, W, C, int(r), float(t), _dtype_code(features), opt,
                                        _p(out_tokens), _p(out_count), _p(out_pos_thw), sp)
         elif workspace is None:
             rc = lib().ttf_compress(_p(features), F, H, W, C, int(r), float(t), _dtype_code(features),
@@ -231,9 +248,9 @@ def ttf_set_match_kernel(which: int = 0) -> None:
         raise TTFError(rc, "ttf_set_match_kernel")
 
 
-def ttf_set_schedule(clips_in_flight: int = 0, l2_mode: int = 0, resident_pct: int = 0) -> None:
-    """ttf_set_schedule: clips of a batch in flight (0 = automatic) and the L2 eviction priorities of the passes."""
-    rc = lib().ttf_set_schedule(int(clips_in_flight), int(l2_mode), int(resident_pct))
+def ttf_set_schedule(clips_in_flight: int = 0) -> None:
+    """ttf_set_schedule: clips of a batch in flight (0 = automatic)."""
+    rc = lib().ttf_set_schedule(int(clips_in_flight))
     if rc != TTF_OK:
         raise TTFError(rc, "ttf_set_schedule")
 
@@ -255,8 +272,10 @@ def ttf_compress_mean(features: torch.Tensor, r: int, t: float, stream=None):
     return out_tokens, out_count, out_pos_thw
 
 
-def ttf_compress_batch(features, r: int, t: float, out_tokens=None, out_count=None, out_pos_thw=None, stream=None):
-    """ttf_compress_batch: `features` is a sequence of [F, H, W, C] device tensors of one shape and dtype.
+def ttf_compress_batch(features, r: int, t: float, out_tokens=None, out_count=None, out_pos_thw=None, stream=None,
+                       anchor_mode: int = 0, anchor_frame: int = 0, order: int = 0, pos_base: int = 0):
+    """ttf_compress_batch (ttf_compress_batch_ex when any option is given): `features` is a sequence of [F, H, W, C]
+    device tensors of one shape and dtype.
     Returns three lists (out_tokens, out_count, out_pos_thw), one entry per clip, as ttf_compress does for one
     clip.  Does not synchronise."""
     feats = list(features)
@@ -277,9 +296,14 @@ def ttf_compress_batch(features, r: int, t: float, out_tokens=None, out_count=No
     if not (len(out_tokens) == len(out_count) == len(out_pos_thw) == B):
         raise ValueError("one output of each kind per clip")
     arr = lambda ts: (ctypes.c_void_p * B)(*[t_.data_ptr() for t_ in ts])
+    opt = _options(anchor_mode, anchor_frame, order, pos_base)
     with torch.cuda.device(dev):
-        rc = lib().ttf_compress_batch(arr(feats), B, F, H, W, C, int(r), float(t), _dtype_code(feats[0]),
-                                      arr(out_tokens), arr(out_count), arr(out_pos_thw), _stream_ptr(stream))
+        if opt is None:
+            rc = lib().ttf_compress_batch(arr(feats), B, F, H, W, C, int(r), float(t), _dtype_code(feats[0]),
+                                          arr(out_tokens), arr(out_count), arr(out_pos_thw), _stream_ptr(stream))
+        else:
+            rc = lib().ttf_compress_batch_ex(arr(feats), B, F, H, W, C, int(r), float(t), _dtype_code(feats[0]), opt,
+                                             arr(out_tokens), arr(out_count), arr(out_pos_thw), _stream_ptr(stream))
     if rc != TTF_OK:
         raise TTFError(rc, "ttf_compress_batch")
     return out_tokens, out_count, out_pos_thw
@@ -303,10 +327,11 @@ def ttf_query(features: torch.Tensor, r: int, t: float, workspace: Optional[torc
             _p(out["dst"]), _p(out["best_sim"]), _p(out["fuse_cnt"])]
     with torch.cuda.device(dev):
         sp = _stream_ptr(stream)
-        if anchor_mode != 0:
+        opt = _options(anchor_mode, anchor_frame, 0, 0)
+        if opt is not None:
             if workspace is not None:
-                raise ValueError("a fixed anchor rule uses the library's own scratch")
-            rc = lib().ttf_query_ex(*args[:8], int(anchor_mode), int(anchor_frame), *args[8:], sp)
+                raise ValueError("the entry point with options uses the library's own scratch")
+            rc = lib().ttf_query_ex(*args[:8], opt, *args[8:], sp)
         elif workspace is None:
             rc = lib().ttf_query(*args, sp)
         else:

@@ -62,16 +62,22 @@ template <typename T, int V, int LS, bool NORMS>
 __global__ void __launch_bounds__(kNormThreads)
 k_norm_sum(const T* __restrict__ X, int F, int N, int C, int nq,
            float* __restrict__ S, float* __restrict__ ssq, int* __restrict__ cnt, int* __restrict__ hdr,
-           int l2_mode, int res_frames, int* __restrict__ tc_cnt, int tc_tiles)
+           int chain)
 {
     using L = Loader<T, V>;
     constexpr int RG = kNormThreads / LS;
     constexpr int WPS = LS / 32;                    // warps across a slice = norm planes per slice
     pdl_launch_dependents();
-    // This kernel may be scheduled while the previous call's gather still runs (it shares the scratch) or
-    // while an upstream kernel still writes X: nothing is read or written before the wait.
-    pdl_wait();
+    // This kernel may be scheduled while the kernel before it in the stream still runs.  Normally that kernel may be
+    // anything (the previous call's gather, which shares the scratch, or an upstream kernel that still writes X), so
+    // nothing is read or written before the wait.  Inside a chain of clips of one batch the predecessor is known: the
+    // gather of the previous clip, which works on another scratch block and another clip; then the sweep runs beside
+    // it, and one CTA waits for it before it exits, so that "this sweep has completed" still implies "everything
+    // before it has completed" for the kernels that follow.  (One CTA, not all: a CTA that waits keeps its place on
+    // the SM, and the CTAs of the sweep that have not started yet need those places.)
+    if (!chain) pdl_wait();
     trace_mark(hdr, 0, false);
+    if (chain) trace_mark(hdr, 15, false);
     const int k = blockIdx.x / nq, q = blockIdx.x - k * nq;
     const int tid = threadIdx.x, lane = tid & 31;
     const int ls = tid & (LS - 1), rg = tid / LS;
@@ -89,15 +95,11 @@ k_norm_sum(const T* __restrict__ X, int F, int N, int C, int nq,
 
     // thread's tokens: rg, rg + RG, rg + 2 RG, ...; a batch is kBatch of them
     typename L::Raw cur[kBatch], nxt[kBatch];
-    // frames the matching pass should still find in L2 keep (or raise) their priority, the others are marked
-    // evict-first so that they do not displace them
-    const uint64_t pol = l2_policy(k < res_frames ? l2_mode : 0);
     auto load_batch = [&](typename L::Raw (&d)[kBatch], int i0) {
 #pragma unroll
         for (int u = 0; u < kBatch; ++u) {
             const int i = i0 + u * RG;
-            d[u] = (active && i < N) ? (l2_mode ? L::load_raw_hint(base + (size_t)i * C, pol) : L::load_raw_cg(base + (size_t)i * C))
-                                     : L::zero();
+            d[u] = (active && i < N) ? L::load_raw_cg(base + (size_t)i * C) : L::zero();
         }
     };
     if (rg < N) load_batch(cur, rg);
@@ -145,8 +147,7 @@ k_norm_sum(const T* __restrict__ X, int F, int N, int C, int nq,
     }
     if (q == 0 && tid == 0) cnt[k] = 0;             // survivor counters start at zero for the matching kernel
     if (blockIdx.x == 0 && tid == 0) hdr[HDR_ERROR] = 0;   // the error word reports on this call only
-    if (blockIdx.x == 0)                            // the tcgen05 matching kernel counts arrivals per tile from zero
-        for (int i = tid; i < tc_tiles; i += kNormThreads) tc_cnt[i] = 0;
+    if (chain && blockIdx.x == 0) pdl_wait();
     trace_mark(hdr, 0, true);
 }
 
@@ -157,9 +158,9 @@ static cudaError_t launch_sum_t(const Problem& p, const Scratch& s, cudaStream_t
     const dim3 g(blocks), b(kNormThreads);
     if (!needs_sweep_norms(p))
         return launch_ex(true, 0, k_norm_sum<T, V, 32, false>, g, b, st, X, p.F, p.N, p.C, p.nq, s.S,
-                         s.ssq, s.cnt, s.hdr, p.l2_mode, p.res_frames, s.tc_cnt, s.tc_tiles);
+                         s.ssq, s.cnt, s.hdr, p.chain);
     return launch_ex(true, 0, k_norm_sum<T, V, 32, true>, g, b, st, X, p.F, p.N, p.C, p.nq, s.S, s.ssq,
-                     s.cnt, s.hdr, p.l2_mode, p.res_frames, s.tc_cnt, s.tc_tiles);
+                     s.cnt, s.hdr, p.chain);
 }
 
 // ---------------------------------------------------------------------------------------------------------

@@ -90,10 +90,8 @@ struct ProfScope {
     }
 };
 
-// Schedule of a batch: clips in flight and the L2 priorities of the passes over X (ttf_set_schedule)
+// Schedule of a batch: clips in flight (ttf_set_schedule)
 static std::atomic<int> g_sched_lanes{0};        // 0: automatic
-static std::atomic<int> g_sched_l2_mode{0};
-static std::atomic<int> g_sched_res_pct{0};
 static std::atomic<int> g_match_kernel{0};       // ttf_set_match_kernel: 0 automatic, 1 warp-level MMA, 2 tcgen05
 
 static size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -115,9 +113,6 @@ void carve_scratch(const Problem& p, void* base, Scratch* s) {
     s->dst = (int*)take(sizeof(int) * FN);
     s->keep = (unsigned char*)take(FN);
     s->fuse_cnt = (int*)take(sizeof(int) * p.N);
-    s->tc_tiles = p.use_tc ? (int)tc_match_tiles(p) : 0;
-    s->tc_cnt = (int*)take(sizeof(int) * (size_t)s->tc_tiles);
-    s->tc_part = (float*)take(sizeof(float) * (p.use_tc ? tc_match_part_floats(p) : 0));
     s->bytes = off;
 }
 
@@ -144,11 +139,10 @@ static int make_problem(const void* X, int F, int H, int W, int C, int r, float 
     p->nslice = p->nq * (p->ls / 32);
     if ((long long)F * p->nq >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
     p->nsl = C % 4 == 0 ? (C + 127) / 128 : (C + 31) / 32;
-    p->anchor_mode = 0; p->anchor_arg = 0; p->emit_anchor = 1; p->pos_t_offset = 0;
-    p->l2_mode = g_sched_l2_mode.load();
-    p->res_frames = (int)(((long long)F * g_sched_res_pct.load() + 99) / 100);
+    p->anchor_mode = 0; p->anchor_arg = 0; p->emit_anchor = 1; p->pos_t_offset = 0; p->pos_base = 0; p->natural_order = 0;
     p->use_tc = 0;
     p->use_tc = (g_match_kernel.load() == 2 && tc_match_eligible(*p)) ? 1 : 0;
+    p->chain = 0; p->chain_next = 0;
     return TTF_OK;
 }
 
@@ -358,6 +352,25 @@ int ttf_workspace_status(const void* workspace, ttf_stream_t stream, int* host_s
     return read_status_words(std::vector<const int*>(1, reinterpret_cast<const int*>(ws)), host_status);
 }
 
+#ifdef TTF_TRACE
+// trace builds only: copies the trace marks (48 64-bit words) of scratch block `block` of the last call on `stream`
+// to host memory and clears them; returns the number of blocks that call used
+int ttf_trace_read(ttf_stream_t stream, int block, unsigned long long* host_out) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    std::lock_guard<std::mutex> lk(g_mu);
+    auto it = g_scratch.find(std::make_pair(dev, (cudaStream_t)stream));
+    if (it == g_scratch.end()) return 0;
+    const int n = (int)it->second.status_words.size();
+    if (block >= 0 && block < n) {
+        const int* hdr = it->second.status_words[block];
+        cudaMemcpy(host_out, hdr + 16, 384, cudaMemcpyDeviceToHost);
+        cudaMemset(const_cast<int*>(hdr) + 16, 0, 384);
+    }
+    return n;
+}
+#endif
+
 int ttf_debug_set_wait(int poll_limit, int tx_extra_bytes) {
     if (poll_limit < 1 || tx_extra_bytes < 0 || tx_extra_bytes % 16 != 0 || tx_extra_bytes > 1024) return TTF_ERR_INVALID_ARG;
     g_wait_limit.store(poll_limit);
@@ -455,13 +468,30 @@ static int set_anchor_rule(Problem* p, int anchor_mode, int anchor_frame) {
     return TTF_OK;
 }
 
+static int set_output_options(Problem* p, int order, int pos_base) {
+    if (order != TTF_ORDER_ANCHOR_FIRST && order != TTF_ORDER_NATURAL) return TTF_ERR_INVALID_ARG;
+    // positions stay inside int32: the largest coordinate is max(F, H, W) - 1 + pos_base
+    const long long top = (long long)(p->F > p->H ? (p->F > p->W ? p->F : p->W) : (p->H > p->W ? p->H : p->W)) + pos_base;
+    if (pos_base < 0 || top >= (1LL << 31)) return TTF_ERR_INVALID_ARG;
+    p->natural_order = order == TTF_ORDER_NATURAL ? 1 : 0;
+    p->pos_base = pos_base;
+    return TTF_OK;
+}
+
+static int apply_options(Problem* p, const ttf_options* opt) {
+    if (!opt) return TTF_OK;
+    int rc = set_anchor_rule(p, opt->anchor_mode, opt->anchor_frame);
+    if (rc == TTF_OK) rc = set_output_options(p, opt->order, opt->pos_base);
+    return rc;
+}
+
 int ttf_compress_ex(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
-                    int anchor_mode, int anchor_frame,
+                    const ttf_options* options,
                     void* out_tokens, int* out_count, int* out_pos_thw, ttf_stream_t stream) {
     if (!features || !out_tokens || !out_count || !out_pos_thw) return TTF_ERR_INVALID_ARG;
     Problem p;
     int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
-    if (rc == TTF_OK) rc = set_anchor_rule(&p, anchor_mode, anchor_frame);
+    if (rc == TTF_OK) rc = apply_options(&p, options);
     if (rc != TTF_OK) return rc;
     Scratch s;
     carve_scratch(p, nullptr, &s);
@@ -472,13 +502,13 @@ int ttf_compress_ex(const void* features, int F, int H, int W, int C, int r, flo
 }
 
 int ttf_query_ex(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
-                 int anchor_mode, int anchor_frame,
+                 const ttf_options* options,
                  int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
                  int* out_fuse_cnt, ttf_stream_t stream) {
     if (!features) return TTF_ERR_INVALID_ARG;
     Problem p;
     int rc = make_problem(features, F, H, W, C, r, t, dtype, &p);
-    if (rc == TTF_OK) rc = set_anchor_rule(&p, anchor_mode, anchor_frame);
+    if (rc == TTF_OK) rc = apply_options(&p, options);
     if (rc != TTF_OK) return rc;
     Scratch s;
     carve_scratch(p, nullptr, &s);
@@ -534,32 +564,57 @@ static int batch_lanes(BatchLanes** out) {
     return TTF_OK;
 }
 
+// The clips of a lane form a chain on the lane's stream: sweep, statistics, matching, gather, next sweep, ... with two
+// scratch blocks used in turn, so that the sweep of a clip can run beside the gather of the clip before it.
 static int batch_on_streams(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
-                            int dtype, void* const* out_tokens, int* const* out_count, int* const* out_pos_thw,
-                            cudaStream_t st) {
+                            int dtype, const ttf_options* options,
+                            void* const* out_tokens, int* const* out_count, int* const* out_pos_thw, cudaStream_t st) {
     std::lock_guard<std::mutex> enqueue(g_lane_mu);
     BatchLanes* L = nullptr;
     int rc = batch_lanes(&L);
     if (rc != TTF_OK) return rc;
+    std::vector<Problem> ps(nclips);
+    size_t stride = 0;
+    for (int n = 0; n < nclips; ++n) {
+        rc = make_problem(features[n], F, H, W, C, r, t, dtype, &ps[n]);
+        if (rc == TTF_OK) rc = apply_options(&ps[n], options);
+        if (rc != TTF_OK) return rc;
+        Scratch s;
+        carve_scratch(ps[n], nullptr, &s);
+        if (s.bytes > stride) stride = s.bytes;
+    }
     int want = g_sched_lanes.load();
-    if (want < 1 || want > kBatchStreams) want = kBatchStreams;
+    if (want < 1 || want > kBatchStreams) want = kBatchStreams;      // automatic: measured best for every clip shape so far
     const int lanes = nclips < want ? nclips : want;
+    std::vector<void*> ws(lanes, nullptr);
+    for (int i = 0; i < lanes; ++i) {            // (may allocate: before the fork, outside the event bracket)
+        rc = cached_scratch(2 * stride, L->s[i], &ws[i]);
+        if (rc != TTF_OK) return rc;
+    }
     cudaError_t e = cudaEventRecord(L->fork, st);
     for (int i = 0; i < lanes && e == cudaSuccess; ++i) e = cudaStreamWaitEvent(L->s[i], L->fork, 0);
     if (e != cudaSuccess) return cuda_fail(e);
     int first_rc = TTF_OK;
-    for (int n = 0; n < nclips && first_rc == TTF_OK; ++n)
-        first_rc = ttf_compress(features[n], F, H, W, C, r, t, dtype, out_tokens[n], out_count[n], out_pos_thw[n],
-                                (ttf_stream_t)L->s[n % lanes]);
+    std::vector<const int*> words;
+    for (int n = 0; n < nclips && first_rc == TTF_OK; ++n) {
+        const int lane = n % lanes, turn = n / lanes;
+        void* block = (char*)ws[lane] + (size_t)(turn & 1) * stride;
+        ps[n].chain = turn > 0 ? 1 : 0;          // the lane's previous kernel is the gather of its previous clip
+        if (turn < 2) {
+            // the block may hold anything (another shape's data, or a failed call's counters): clear its control words
+            first_rc = clear_control(ps[n], block, L->s[lane]);
+            words.push_back(reinterpret_cast<const int*>(block));
+            if (first_rc != TTF_OK) break;
+            if (turn == 1) ps[n].chain = 0;      // (the memset sits between the gather and this sweep)
+        }
+        // (the lane's next clip, if there is one, is at turn + 1; its sweep is chained from turn 2 on)
+        ps[n].chain_next = (n + lanes < nclips && turn + 1 >= 2) ? 1 : 0;
+        first_rc = compress_impl(ps[n], block, out_tokens[n], out_count[n], out_pos_thw[n], L->s[lane]);
+    }
     {   // the caller asks about the batch through its own stream: point it at the lanes' error words
         int dev = 0;
-        std::vector<const int*> words;
         if (cudaGetDevice(&dev) == cudaSuccess) {
             std::lock_guard<std::mutex> lk(g_mu);
-            for (int i = 0; i < lanes; ++i) {
-                auto it = g_scratch.find(std::make_pair(dev, L->s[i]));
-                if (it != g_scratch.end()) words.insert(words.end(), it->second.status_words.begin(), it->second.status_words.end());
-            }
             g_scratch[std::make_pair(dev, st)].status_words = words;
         }
     }
@@ -579,12 +634,9 @@ int ttf_set_match_kernel(int which) {
     return TTF_OK;
 }
 
-int ttf_set_schedule(int clips_in_flight, int l2_mode, int resident_pct) {
-    if (clips_in_flight < 0 || clips_in_flight > kBatchStreams || l2_mode < 0 || l2_mode > 2 || resident_pct < 0 ||
-        resident_pct > 100) return TTF_ERR_INVALID_ARG;
+int ttf_set_schedule(int clips_in_flight) {
+    if (clips_in_flight < 0 || clips_in_flight > kBatchStreams) return TTF_ERR_INVALID_ARG;
     g_sched_lanes.store(clips_in_flight);
-    g_sched_l2_mode.store(l2_mode);
-    g_sched_res_pct.store(resident_pct);
     return TTF_OK;
 }
 
@@ -598,7 +650,17 @@ int ttf_compress_batch(const void* const* features, int nclips, int F, int H, in
     Problem p;
     int rc = make_problem(features[0], F, H, W, C, r, t, dtype, &p);
     if (rc != TTF_OK) return rc;
-    return batch_on_streams(features, nclips, F, H, W, C, r, t, dtype, out_tokens, out_count, out_pos_thw, st);
+    return batch_on_streams(features, nclips, F, H, W, C, r, t, dtype, nullptr, out_tokens, out_count, out_pos_thw, st);
+}
+
+int ttf_compress_batch_ex(const void* const* features, int nclips, int F, int H, int W, int C, int r, float t,
+                          int dtype, const ttf_options* options,
+                          void* const* out_tokens, int* const* out_count, int* const* out_pos_thw, ttf_stream_t stream) {
+    if (!features || !out_tokens || !out_count || !out_pos_thw || nclips < 1) return TTF_ERR_INVALID_ARG;
+    for (int n = 0; n < nclips; ++n)
+        if (!features[n] || !out_tokens[n] || !out_count[n] || !out_pos_thw[n]) return TTF_ERR_INVALID_ARG;
+    return batch_on_streams(features, nclips, F, H, W, C, r, t, dtype, options, out_tokens, out_count, out_pos_thw,
+                            (cudaStream_t)stream);
 }
 
 int ttf_compress_segment(const void* features, int F, int H, int W, int C, int r, float t, int dtype,

@@ -46,11 +46,13 @@ __device__ __forceinline__ void fuse_count_cta(int F, int H, int W, int r, int a
     }
 }
 
-// Frame search of the gather: the frame that holds the e-th preserved source token (flat order, anchor frame
-// skipped) and the number of preserved tokens before that frame.  Returns the total P; k_out = -1 when e is past
-// the end (e < 0 asks for the total only).  All lanes of a warp call it with the same arguments.
+// Frame search of the gather: the frame that holds the e-th token of the flat walk and the number of walked tokens
+// before that frame.  The walk visits the preserved tokens of the source frames in flat order; the anchor frame
+// contributes `acnt` tokens: 0 when its rows are emitted as a block of their own (Eq. xprime_stack), N in natural
+// order (all of its tokens are retained, Eq. mask).  Returns the total; k_out = -1 when e is past the end (e < 0
+// asks for the total only).  All lanes of a warp call it with the same arguments.
 __device__ __forceinline__ int find_frame(const int* __restrict__ cnt, const int* __restrict__ gprefix, int F, int a,
-                                          int lane, int e, int& k_out, int& before) {
+                                          int acnt, int lane, int e, int& k_out, int& before) {
     int running = 0;
     k_out = -1; before = 0;
     if (F > kWarpPrefixMaxF) {                         // pre-scanned prefix: binary search
@@ -67,7 +69,7 @@ __device__ __forceinline__ int find_frame(const int* __restrict__ cnt, const int
 #pragma unroll
         for (int q = 0; q < kScanChunks; ++q) {
             const int k = base + q * 32 + lane;
-            c[q] = (k < F && k != a) ? __ldcg(cnt + k) : 0;
+            c[q] = k < F ? (k == a ? acnt : __ldcg(cnt + k)) : 0;
         }
 #pragma unroll
         for (int q = 0; q < kScanChunks; ++q) {

@@ -10,15 +10,14 @@ namespace ttf {
 
 constexpr float kNormFloor = 1e-12f;   // norms are floored here before dividing (zero token -> similarity 0)
 constexpr int kWarpPrefixMaxF = 1024;  // frame counts up to this are scanned by each warp of the gather itself
-constexpr int kHdrInts = 64;
+constexpr int kHdrInts = 128;
 constexpr int kStatReplicas = 16;      // copies of the frame statistics, so that the CTAs that read them at the
                                        // same moment do not all queue on the same few cache lines
 
 // header words of the scratch block
 enum { HDR_ANCHOR = 0,          // anchor frame a*
        HDR_DONE_ALL = 1,        // arrival counter of the statistics CTAs (zero between calls)
-       HDR_ERROR = 2,           // a bounded wait of this call gave up (cleared by the first kernel of every call)
-       HDR_GATHER_DONE = 3 };   // arrival counter of the gather's warps (zero between calls)
+       HDR_ERROR = 2 };         // a bounded wait of this call gave up (cleared by the first kernel of every call)
 
 // Problem description handed to every launcher.
 struct Problem {
@@ -37,10 +36,12 @@ struct Problem {
     int anchor_arg;     // explicit anchor frame
     int emit_anchor;    // 1: X' starts with the N anchor rows (Eq. xprime_stack); 0: streaming segment, sources only
     int pos_t_offset;   // added to the frame coordinate of every emitted position
-    int l2_mode;        // L2 eviction priorities of the passes over X: 0 none; 1: frames < res_frames default priority,
-                        // everything else evict-first; 2: frames < res_frames evict-last, everything else evict-first
-    int res_frames;     // leading frames of the clip that the sweep asks L2 to keep for the matching pass
-    int use_tc;         // 1: the matching step runs on tcgen05 (ttf_match_tc.cu), norms from the sweep
+    int pos_base;       // added to all three coordinates of every emitted position
+    int natural_order;  // 1: all retained tokens in ascending flat index (the anchor rows where they fall)
+    int use_tc;         // 1: the matching step runs on tcgen05 (ttf_match_tc.cu)
+    int chain;          // 1: the kernel before this call's sweep in the stream is the gather of the library's previous
+                        // clip, which works on another scratch block: the sweep may run beside it
+    int chain_next;     // 1: the kernel after this call's gather is such a sweep
 };
 
 // Device pointers carved out of one scratch allocation.
@@ -57,9 +58,6 @@ struct Scratch {
     int* dst;           // [F*N] best anchor cell (Eq. dst)
     unsigned char* keep;// [F*N] retention mask (Eq. mask)
     int* fuse_cnt;      // [N]   tokens fused into each anchor cell
-    float* tc_part;     // tcgen05 matching: partial window sums [tile][piece][(2r+1)^2][128] (pieces > 1 only)
-    int* tc_cnt;        // tcgen05 matching: arrival counter per tile (zero between calls)
-    int tc_tiles;       // number of those counters
     size_t bytes;       // total, multiple of 256
 };
 
@@ -84,12 +82,11 @@ inline bool uses_mma_match(const Problem& p) {
 }
 
 // The sweep stores per-token partial squared norms only for the kernels that read them.
-inline bool needs_sweep_norms(const Problem& p) { return !uses_mma_match(p) || p.r == 2 || p.use_tc; }
+inline bool needs_sweep_norms(const Problem& p) { return !p.use_tc && (!uses_mma_match(p) || p.r == 2); }
 
 // tcgen05 matching (ttf_match_tc.cu)
 bool tc_match_eligible(const Problem& p);
 int tc_match_pieces(const Problem& p);
-size_t tc_match_part_floats(const Problem& p);
 size_t tc_match_tiles(const Problem& p);
 cudaError_t launch_match_tc(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                             unsigned char* keep, cudaStream_t st);
@@ -176,35 +173,37 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, c
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// Development aid (compiled out unless TTF_TRACE is defined): earliest start / latest end of every kernel of
-// a call in nanoseconds of the global timer, kept in header words 16..47 of the scratch block.
+// Development aid (compiled out unless the library is built with -DTTF_TRACE): earliest / latest time at which
+// any CTA passed a mark, in nanoseconds of the global timer, kept in header words 16..111 of the scratch block
+// (mark id < 24; two 64-bit words each: ~earliest, latest).  trace_mark is called by thread 0 of a CTA,
+// trace_mark_any by whichever single thread reaches the point.
 #ifdef TTF_TRACE
+__device__ __forceinline__ void trace_mark_any(int* hdr, int id, bool end) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    unsigned long long* s = reinterpret_cast<unsigned long long*>(hdr + 16) + id * 2 + (end ? 1 : 0);
+    atomicMax(s, end ? t : ~t);
+}
 __device__ __forceinline__ void trace_mark(int* hdr, int id, bool end) {
-    if (threadIdx.x == 0) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        unsigned long long* s = reinterpret_cast<unsigned long long*>(hdr + 16) + id * 2 + (end ? 1 : 0);
-        atomicMax(s, end ? t : ~t);
-    }
+    if (threadIdx.x == 0) trace_mark_any(hdr, id, end);
+}
+// mean of a duration over the threads that report it: word 0 of the mark = sum of nanoseconds, word 1 = reports
+__device__ __forceinline__ unsigned long long trace_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void trace_acc(int* hdr, int id, unsigned long long ns) {
+    unsigned long long* s = reinterpret_cast<unsigned long long*>(hdr + 16) + id * 2;
+    atomicAdd(s, ns);
+    atomicAdd(s + 1, 1ull);
 }
 #else
+__device__ __forceinline__ void trace_mark_any(int*, int, bool) {}
 __device__ __forceinline__ void trace_mark(int*, int, bool) {}
+__device__ __forceinline__ unsigned long long trace_now() { return 0; }
+__device__ __forceinline__ void trace_acc(int*, int, unsigned long long) {}
 #endif
-
-// L2 eviction-priority policies (createpolicy) and 16-byte loads that carry one
-__device__ __forceinline__ uint64_t l2_policy(int kind) {     // 0 evict_first, 1 evict_normal, 2 evict_last
-    uint64_t p;
-    if (kind == 0) asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    else if (kind == 2) asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-    else asm volatile("createpolicy.fractional.L2::evict_normal.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ uint4 ldcg_hint16(const void* p, uint64_t pol) {
-    uint4 v;
-    asm volatile("ld.global.cg.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
-    return v;
-}
 
 struct bf16_t { uint16_t bits; };   // storage type only: all arithmetic is on the widened fp32 value
 
@@ -218,10 +217,6 @@ template <> struct Loader<float, 4> {
     using Raw = float4;
     static __device__ __forceinline__ Raw load_raw(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
     static __device__ __forceinline__ Raw load_raw_cg(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
-    static __device__ __forceinline__ Raw load_raw_hint(const float* p, uint64_t pol) {
-        const uint4 v = ldcg_hint16(p, pol);
-        return make_float4(__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w));
-    }
     static __device__ __forceinline__ Raw zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[4]) { x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
     static __device__ __forceinline__ void load(const float* p, float (&x)[4]) { unpack(load_raw(p), x); }
@@ -230,7 +225,6 @@ template <> struct Loader<float, 1> {
     using Raw = float;
     static __device__ __forceinline__ Raw load_raw(const float* p) { return __ldg(p); }
     static __device__ __forceinline__ Raw load_raw_cg(const float* p) { return __ldcg(p); }
-    static __device__ __forceinline__ Raw load_raw_hint(const float* p, uint64_t) { return __ldcg(p); }
     static __device__ __forceinline__ Raw zero() { return 0.f; }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[1]) { x[0] = v; }
     static __device__ __forceinline__ void load(const float* p, float (&x)[1]) { x[0] = __ldg(p); }
@@ -239,7 +233,6 @@ template <> struct Loader<bf16_t, 8> {
     using Raw = uint4;
     static __device__ __forceinline__ Raw load_raw(const bf16_t* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
     static __device__ __forceinline__ Raw load_raw_cg(const bf16_t* p) { return __ldcg(reinterpret_cast<const uint4*>(p)); }
-    static __device__ __forceinline__ Raw load_raw_hint(const bf16_t* p, uint64_t pol) { return ldcg_hint16(p, pol); }
     static __device__ __forceinline__ Raw zero() { return make_uint4(0, 0, 0, 0); }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[8]) {
         x[0] = bf16_lo(v.x); x[1] = bf16_hi(v.x); x[2] = bf16_lo(v.y); x[3] = bf16_hi(v.y);
@@ -255,7 +248,6 @@ template <> struct Loader<bf16_t, 1> {
     static __device__ __forceinline__ Raw load_raw_cg(const bf16_t* p) {
         return __uint_as_float(static_cast<uint32_t>(__ldcg(reinterpret_cast<const unsigned short*>(p))) << 16);
     }
-    static __device__ __forceinline__ Raw load_raw_hint(const bf16_t* p, uint64_t) { return load_raw_cg(p); }
     static __device__ __forceinline__ Raw zero() { return 0.f; }
     static __device__ __forceinline__ void unpack(const Raw& v, float (&x)[1]) { x[0] = v; }
     static __device__ __forceinline__ void load(const bf16_t* p, float (&x)[1]) { x[0] = load_raw(p); }

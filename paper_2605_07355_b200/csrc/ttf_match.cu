@@ -93,7 +93,7 @@ template <int MT, int NT, bool GRAM, int ST>
 __device__ __forceinline__ void match_mma_body(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t,
                                                const AnchorSrc& asrc, const float* ssq, int nslice,
                                                float* __restrict__ shat, int* __restrict__ dst,
-                                               unsigned char* __restrict__ keep, int* __restrict__ cnt, int l2_mode)
+                                               unsigned char* __restrict__ keep, int* __restrict__ cnt)
 {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     const int N = H * W;
@@ -115,7 +115,7 @@ __device__ __forceinline__ void match_mma_body(const bf16_t* __restrict__ X, int
         trace_mark(asrc.hdr, 4, true);
         return a;
     };
-    match_mma_unit<MT, NT, GRAM, ST>(X, F, H, W, C, r, t, anchor_fn, i, k0, ssq, nslice, shat, dst, keep, cnt, dyn_smem, l2_mode);
+    match_mma_unit<MT, NT, GRAM, ST>(X, F, H, W, C, r, t, anchor_fn, i, k0, ssq, nslice, shat, dst, keep, cnt, dyn_smem);
     trace_mark(asrc.hdr, 2, true);
 }
 
@@ -123,10 +123,9 @@ __device__ __forceinline__ void match_mma_body(const bf16_t* __restrict__ X, int
 template <int MT, int NT>
 __global__ void TTF_MMA_BOUNDS
 k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t, AnchorSrc asrc,
-            float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt,
-            int l2_mode)
+            float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt)
 {
-    match_mma_body<MT, NT, true, kMmaStagesDefault>(X, F, H, W, C, r, t, asrc, nullptr, 0, shat, dst, keep, cnt, l2_mode);
+    match_mma_body<MT, NT, true, kMmaStagesDefault>(X, F, H, W, C, r, t, asrc, nullptr, 0, shat, dst, keep, cnt);
 }
 
 // r = 2: the 25 candidate rows of a cell are as much data as 25 source rows, so a CTA takes 64 frames per cell to
@@ -143,10 +142,9 @@ constexpr int kWideStages = TTF_WIDE_STAGES;
 __global__ void __launch_bounds__(kMmaWarps * 32, 2)
 k_match_mma_wide(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t, AnchorSrc asrc,
                  const float* __restrict__ ssq, int nslice,
-                 float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt,
-                 int l2_mode)
+                 float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt)
 {
-    match_mma_body<kWideMT, 4, false, kWideStages>(X, F, H, W, C, r, t, asrc, ssq, nslice, shat, dst, keep, cnt, l2_mode);
+    match_mma_body<kWideMT, 4, false, kWideStages>(X, F, H, W, C, r, t, asrc, ssq, nslice, shat, dst, keep, cnt);
 }
 
 template <int MT, int NT>
@@ -158,7 +156,7 @@ static cudaError_t launch_mma_t(const Problem& p, const Scratch& s, int* out_anc
     if (e != cudaSuccess) return e;
     return launch_ex(true, smem, k_match_mma<MT, NT>, dim3((unsigned)(chunks * p.N)),
                      dim3(kMmaWarps * 32), st, reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t,
-                     make_anchor_src(p, s, out_anchor), shat, dst, keep, s.cnt, p.l2_mode);
+                     make_anchor_src(p, s, out_anchor), shat, dst, keep, s.cnt);
 }
 
 static cudaError_t launch_mma_wide(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
@@ -169,7 +167,7 @@ static cudaError_t launch_mma_wide(const Problem& p, const Scratch& s, int* out_
     const long long chunks = (p.F + 16 * kWideMT - 1) / (16 * kWideMT);
     return launch_ex(true, smem, k_match_mma_wide, dim3((unsigned)(chunks * p.N)), dim3(kMmaWarps * 32),
                      st, reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t,
-                     make_anchor_src(p, s, out_anchor), (const float*)s.ssq, p.nslice, shat, dst, keep, s.cnt, p.l2_mode);
+                     make_anchor_src(p, s, out_anchor), (const float*)s.ssq, p.nslice, shat, dst, keep, s.cnt);
 }
 
 template <typename T, int V>

@@ -49,12 +49,6 @@ __device__ __forceinline__ void cp_async16(void* dst_smem, const void* src, bool
     const int bytes = valid ? 16 : 0;            // 0 source bytes: the 16 destination bytes are zero-filled
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
 }
-// the same with an L2 eviction-priority policy for the source line
-__device__ __forceinline__ void cp_async16_hint(void* dst_smem, const void* src, bool valid, uint64_t pol) {
-    const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(dst_smem));
-    const int bytes = valid ? 16 : 0;
-    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;" ::"r"(d), "l"(src), "r"(bytes), "l"(pol) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
@@ -63,17 +57,14 @@ template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile(
 template <int MT, int NT, bool DO_A = true, bool DO_B = true>
 __device__ __forceinline__ void mma_issue_stage(uint4* slot, const uint4* const (&arow)[MT][2],
                                                 const uint4* const (&brow)[NT], const bool (&bvalid)[NT],
-                                                int idx, int units, int lane, bool hint = false, uint64_t pol_a = 0) {
+                                                int idx, int units, int lane) {
     const bool ok = idx < units;
     const int safe = ok ? idx : 0;
     if constexpr (DO_A) {
 #pragma unroll
         for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                if (hint) cp_async16_hint(slot + (mt * 2 + h) * 32 + lane, arow[mt][h] + safe, ok, pol_a);
-                else cp_async16(slot + (mt * 2 + h) * 32 + lane, arow[mt][h] + safe, ok);
-            }
+            for (int h = 0; h < 2; ++h) cp_async16(slot + (mt * 2 + h) * 32 + lane, arow[mt][h] + safe, ok);
     }
     if constexpr (DO_B) {
 #pragma unroll
@@ -134,7 +125,7 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
                                                AnchorFn anchor_fn, int i, int k0, const float* ssq, int nslice,
                                                float* __restrict__ shat, int* __restrict__ dst,
                                                unsigned char* __restrict__ keep, int* __restrict__ cnt,
-                                               unsigned char* dyn_smem, int l2_mode = 0)
+                                               unsigned char* dyn_smem)
 {
     constexpr int kMmaStages = ST;
     constexpr int FR = 16 * MT;      // frames per CTA
@@ -157,9 +148,6 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
     const int g = lane >> 2, tig = lane & 3;
     const int y = i / W, x = i - y * W;
     const int side = 2 * r + 1, ncand = side * side;
-    // source rows are read for the last time but for the gather of the preserved third: evict-first
-    const bool hint = l2_mode != 0;
-    const uint64_t pol_a = l2_policy(0);
     const int units = C / 8;                     // 16-byte units per row
 
     // candidate c = (dy + r) * side + (dx + r): ascending c is ascending anchor index among in-grid cells
@@ -191,7 +179,7 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
     for (int st = 0; st < kMmaStages - 1; ++st)
         if (st < nmine)
             mma_issue_stage<MT, NT, true, false>(wring + st * PIECES * 32, arow, brow, bvalid,
-                                                 (w + st * kMmaWarps) * 4 + tig, units, lane, hint, pol_a);
+                                                 (w + st * kMmaWarps) * 4 + tig, units, lane);
     cp_async_commit();
 
     const int a = anchor_fn();
@@ -237,7 +225,7 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
         const int nb = b + kMmaStages - 1;
         if (nb < nmine)
             mma_issue_stage<MT, NT>(wring + (nb % kMmaStages) * PIECES * 32, arow, brow, bvalid,
-                                    (w + nb * kMmaWarps) * 4 + tig, units, lane, hint, pol_a);
+                                    (w + nb * kMmaWarps) * 4 + tig, units, lane);
         cp_async_commit();
         cp_async_wait<kMmaStages - 1>();         // block b has landed (each lane waits for its own copies)
         mma_consume_stage<MT, NT, GRAM>(wring + (b % kMmaStages) * PIECES * 32, lane, acc, accn, accb);

@@ -15,11 +15,14 @@
 //   Both arrive with the 128-byte swizzle, which is the K-major operand layout of tcgen05.mma; a pipeline stage is
 //   64 channels (4 MMAs of K = 16).  fp32 accumulation in tensor memory; bf16 products are exact in fp32.
 //
-// The channel range of a tile is cut into `pieces` consecutive parts, one CTA each, so that a clip gives at least
-// two CTAs per SM; the partial sums of a tile go through global memory and are added in piece order by whichever
-// CTA of the tile arrives last (an arrival counter per tile), so the result does not depend on scheduling.
-// Token norms come from the sweep's partial squared norms.  Warp roles: 0 TMA producer, 1 tensor-memory owner and
-// MMA issuer, 2-5 epilogue (one tensor-memory lane = one source row per thread).
+// The channel range of a tile is cut into `pieces` consecutive parts, one CTA each, so that a small clip still gives
+// about two CTAs per SM.  The CTAs of a tile form a thread-block cluster: when their pipelines have drained, ranks
+// > 0 write their partial sums into rank 0's shared memory (distributed shared memory, two cluster barriers) and
+// rank 0 adds them in rank order, so the result does not depend on scheduling.
+// Token norms are taken from the tiles themselves: while the pipeline runs, every epilogue thread adds up the squares
+// of "its" source row (and the first NCAND threads those of a candidate row) as the stages pass through shared memory.
+// Warp roles: 0 TMA producer, 1 tensor-memory owner and MMA issuer, 2-5 epilogue (one tensor-memory lane = one
+// source row per thread).
 //
 // Every mbarrier wait is bounded; a wait that runs out sets the error word of the call, the CTA stops feeding its
 // pipeline, waits (bounded again) for the copies it has in flight, frees its tensor memory and returns.
@@ -120,11 +123,37 @@ template <int R> struct TcShape {
     static constexpr int WIN = SIDE * SIDE;               // candidates of one source row
 };
 
+// ---- thread-block clusters: the CTAs of one tile exchange their partial sums through distributed shared memory
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// all threads of all CTAs of the cluster; writes before it are visible to every CTA of the cluster after it
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t local_smem_addr, uint32_t rank, float v) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_smem_addr), "r"(rank));
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+}
+
+// sum of squares of the 8 bf16 values of a 16-byte piece
+__device__ __forceinline__ float ssq8(const uint4& v, float acc) {
+    float x;
+    x = bf16_lo(v.x); acc = fmaf(x, x, acc); x = bf16_hi(v.x); acc = fmaf(x, x, acc);
+    x = bf16_lo(v.y); acc = fmaf(x, x, acc); x = bf16_hi(v.y); acc = fmaf(x, x, acc);
+    x = bf16_lo(v.z); acc = fmaf(x, x, acc); x = bf16_hi(v.z); acc = fmaf(x, x, acc);
+    x = bf16_lo(v.w); acc = fmaf(x, x, acc); x = bf16_hi(v.w); acc = fmaf(x, x, acc);
+    return acc;
+}
+
 template <int R>
 __global__ void __launch_bounds__(kTcThreads)
 k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
-           int F, int H, int W, int C, float t, AnchorSrc asrc, const float* __restrict__ ssq, int nslice,
-           int pieces, float* __restrict__ part, int* __restrict__ tile_cnt,
+           int F, int H, int W, int C, float t, AnchorSrc asrc, int pieces,
            float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt,
            int wait_limit)
 {
@@ -132,13 +161,15 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
     extern __shared__ unsigned char dyn_raw[];
     __shared__ uint64_t bar_full[S::STAGES], bar_empty[S::STAGES], bar_acc;
     __shared__ uint32_t s_tmem;
-    __shared__ int s_err, s_last;
-    __shared__ float s_ra[S::NCAND];
+    __shared__ int s_err;
+    __shared__ float s_nb[S::NCAND];                       // squared norms of the candidate rows
+    __shared__ float s_nbp[S::NCAND * 8];                  // ... per 16-byte piece column, before they are added up
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = H * W;
     const int xs_n = (W + kTcWB - 1) / kTcWB;
-    const int tile = blockIdx.x / pieces, piece = blockIdx.x - tile * pieces;
+    const int tile = blockIdx.x / pieces;
+    const int piece = pieces > 1 ? (int)cluster_rank() : 0;        // = blockIdx.x % pieces
     const int kg = tile / (H * xs_n), rem = tile - kg * (H * xs_n);
     const int y = rem / xs_n, x0 = (rem - y * xs_n) * kTcWB;
     const int k0 = kg * kTcFR;
@@ -151,11 +182,14 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
     unsigned char* dyn = dyn_raw + (dyn_base - smem_u32(dyn_raw));
 
     pdl_launch_dependents();
+    trace_mark(asrc.hdr, 2, false);
     if (tid == 0) {
-        for (int s = 0; s < S::STAGES; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 1); }
+        // a stage is full when its two copies have landed, and free again when the MMAs that read it have completed
+        // and each of the four epilogue warps has taken its share of the norms from it
+        for (int s = 0; s < S::STAGES; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 5); }
         mbar_init(&bar_acc, 1);
         mbar_init_fence();
-        s_err = 0; s_last = 0;
+        s_err = 0;
         tensormap_prefetch(&mapA);
         tensormap_prefetch(&mapB);
     }
@@ -171,13 +205,22 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
     tc_fence_after();
     const uint32_t tmem = s_tmem;
 
-    // everything upstream (the sweep's norms, the anchor, and whatever produced X) is complete after this wait
+    // everything upstream (the anchor, and whatever produced X) is complete after this wait
+    trace_mark(asrc.hdr, 11, false); trace_mark(asrc.hdr, 11, true);     // set-up done
     pdl_wait();
+    trace_mark(asrc.hdr, 5, false);
     const int a = asrc.fixed >= 0 ? asrc.fixed : __ldcg(asrc.hdr + HDR_ANCHOR);
     if (blockIdx.x == 0 && tid == 0 && asrc.fixed >= 0) {
         asrc.hdr[HDR_ANCHOR] = a;                // the gather reads it from here
         if (asrc.out_anchor) *asrc.out_anchor = a;
     }
+
+    // epilogue-thread state that outlives the role code
+    const int q = warp & 3;                                // tensor-memory lane quadrant an epilogue warp may read
+    const int m = q * 32 + lane;                           // source row of an epilogue thread: 4 * frame + cell
+    const int et = (warp - 2) * 32 + lane;                 // 0..127 among the epilogue threads
+    float win[S::WIN];                                     // this row's window of dot products
+    float na = 0.f, nb = 0.f;                              // squared norm of source row m / of candidate row et
 
     if (warp == 0) {
         // ---- producer: one lane issues the tile copies of every stage ----------------------------------------
@@ -194,6 +237,7 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
                 tma_load_4d(sa + kTcABytes, &mapB, c0, x0 - R, y - R, a, &bar_full[s]);
                 issued = it + 1;
             }
+            trace_mark_any(asrc.hdr, 12, false); trace_mark_any(asrc.hdr, 12, true);   // all copies issued
             if (*(volatile int*)&s_err) {
                 // copies already issued still land in this CTA's shared memory: wait (bounded) for the stages that
                 // nobody consumed before the CTA is allowed to exit
@@ -205,38 +249,67 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
         // ---- MMA issuer: one lane, four K = 16 steps per stage -----------------------------------------------
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_bf16(S::NB);
-            bool ok = true;
-            for (int it = 0; it < nst && ok; ++it) {
+            for (int it = 0; it < nst; ++it) {
                 const int s = it % S::STAGES;
-                if (!mbar_wait(&bar_full[s], (it / S::STAGES) & 1, wait_limit)) { atomicExch(&s_err, 1); ok = false; break; }
+                if (!mbar_wait(&bar_full[s], (it / S::STAGES) & 1, wait_limit)) { atomicExch(&s_err, 1); break; }
                 tc_fence_after();
                 const uint32_t sa = dyn_base + (uint32_t)s * S::STAGE;
                 const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + kTcABytes);
 #pragma unroll
                 for (int k = 0; k < kTcKC / 16; ++k)       // 32 bytes further along K inside the swizzle row
                     umma_bf16(tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, it > 0 || k > 0);
-                umma_commit(&bar_empty[s]);                // the stage is free once these MMAs have read it
+                umma_commit(&bar_empty[s]);                // one of the five arrivals that free the stage
             }
             umma_commit(&bar_acc);                         // accumulator complete (also arrives after a give-up)
         }
     } else {
-        // ---- epilogue: thread = source row m = 4 * frame + cell ----------------------------------------------
-        const int q = warp & 3;                            // tensor-memory lane quadrant this warp may read
-        const int m = q * 32 + lane;
-        const int et = (warp - 2) * 32 + lane;             // 0..127 among the epilogue threads
-        const int kl = m >> 2, dx = m & 3;
-        const int k = k0 + kl, x = x0 + dx;
-        const bool row_ok = k < F && x < W;
-        const size_t FN = (size_t)F * N;
-        const size_t f = (size_t)(row_ok ? k : 0) * N + (size_t)y * W + (row_ok ? x : 0);
-        // inverse norms (independent of the accumulator: fetched while the pipeline runs)
-        const float rs = row_ok ? inv_norm(ssq, nslice, FN, f) : 0.f;
-        if (et < S::NCAND) {
-            const int yy = y - R + et / S::BW, xx = x0 - R + et % S::BW;
-            s_ra[et] = (yy >= 0 && yy < H && xx >= 0 && xx < W) ? inv_norm(ssq, nslice, FN, (size_t)a * N + (size_t)yy * W + xx) : 0.f;
+        // ---- epilogue warps, part 1: while the pipeline runs, the squared norms of the rows that pass through
+        // shared memory (source row m by every thread, candidate row et by the first NCAND threads).  A row is 128
+        // bytes per stage; its 16-byte pieces sit at (piece ^ (row & 7)) (the 128-byte swizzle), and a sum of
+        // squares does not care in which order it meets them ---------------------------------------------------
+        bool ok = true;
+        constexpr int NP = S::NCAND * 8;                   // (candidate row, 16-byte piece column) pairs
+        constexpr int PP = (NP + 127) / 128;               // pairs per epilogue thread
+        float na8[8], nbq[PP];                             // one running sum per piece column: eight short chains
+#pragma unroll
+        for (int c = 0; c < 8; ++c) na8[c] = 0.f;
+#pragma unroll
+        for (int u = 0; u < PP; ++u) nbq[u] = 0.f;
+        for (int it = 0; it < nst; ++it) {
+            const int s = it % S::STAGES;
+            if (!mbar_wait(&bar_full[s], (it / S::STAGES) & 1, wait_limit)) { atomicExch(&s_err, 1); ok = false; break; }
+            const unsigned char* sa = dyn + (size_t)s * S::STAGE;
+            const uint4* rowa = reinterpret_cast<const uint4*>(sa + (size_t)m * 128);
+            uint4 va[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) va[c] = rowa[c ^ (m & 7)];
+            uint4 vb[PP];
+#pragma unroll
+            for (int u = 0; u < PP; ++u) {
+                const int pr = et + u * 128, row = pr >> 3, pc = pr & 7;
+                vb[u] = pr < NP ? reinterpret_cast<const uint4*>(sa + kTcABytes + (size_t)row * 128)[pc ^ (row & 7)]
+                                : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c) na8[c] = ssq8(va[c], na8[c]);
+#pragma unroll
+            for (int u = 0; u < PP; ++u) nbq[u] = ssq8(vb[u], nbq[u]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar_empty[s]);
         }
-        bool ok = mbar_wait(&bar_acc, 0, wait_limit);
+        na = ((na8[0] + na8[1]) + (na8[2] + na8[3])) + ((na8[4] + na8[5]) + (na8[6] + na8[7]));
+#pragma unroll
+        for (int u = 0; u < PP; ++u) if (et + u * 128 < NP) s_nbp[et + u * 128] = nbq[u];
+        epilogue_bar_sync();
+        if (et < S::NCAND) {
+            const float* pp = s_nbp + et * 8;
+            nb = ((pp[0] + pp[1]) + (pp[2] + pp[3])) + ((pp[4] + pp[5]) + (pp[6] + pp[7]));
+        }
+        if (et == 0) { trace_mark_any(asrc.hdr, 13, false); trace_mark_any(asrc.hdr, 13, true); }   // norms done
+        // ---- part 2: the accumulator ---------------------------------------------------------------------------
+        if (ok) ok = mbar_wait(&bar_acc, 0, wait_limit);
         if (!ok) atomicExch(&s_err, 1);
+        if (et == 0) { trace_mark_any(asrc.hdr, 14, false); trace_mark_any(asrc.hdr, 14, true); }   // accumulator complete
         tc_fence_after();
         float d[S::NB];
         if (ok) {
@@ -252,7 +325,7 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
             for (int i = 0; i < S::NB; ++i) d[i] = 0.f;
         }
         // this row's window: candidate (dy, ddx) is column (dy + R) * BW + dx + ddx + R of the tile
-        float win[S::WIN];
+        const int dx = m & 3;
 #pragma unroll
         for (int wy = 0; wy < S::SIDE; ++wy)
 #pragma unroll
@@ -260,35 +333,47 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
                 const int n0 = wy * S::BW + wx;
                 win[wy * S::SIDE + wx] = dx == 0 ? d[n0] : (dx == 1 ? d[n0 + 1] : (dx == 2 ? d[n0 + 2] : d[n0 + 3]));
             }
-        bool last = true;
-        if (pieces > 1) {
-            // partial sums of this piece: [tile][piece][candidate][row], rows contiguous across the threads
-            float* mine = part + ((size_t)blockIdx.x * S::WIN) * kTcM + m;
+    }
+
+    // ---- split K: the CTAs of a tile form a cluster; ranks > 0 hand their partial sums to rank 0 through its
+    // shared memory (the stage ring, idle by then) and rank 0 adds them in rank order ----------------------------
+    constexpr int XROW = (S::WIN + 1) * kTcM + S::NCAND;   // floats one rank sends: window sums, row norms, candidate norms
+    if (pieces > 1) {
+        __syncwarp();
+        cluster_sync_all();                                // every CTA of the tile is past its pipeline: rank 0's ring is idle
+        if (warp >= 2 && piece > 0) {
+            const uint32_t base = dyn_base + (uint32_t)(piece - 1) * XROW * 4;
 #pragma unroll
-            for (int c = 0; c < S::WIN; ++c) __stcg(mine + (size_t)c * kTcM, win[c]);
-            __threadfence();
-            epilogue_bar_sync();
-            if (et == 0) s_last = atomicAdd(tile_cnt + tile, 1) == pieces - 1;
-            epilogue_bar_sync();
-            last = s_last != 0;
-            if (last) {
-                __threadfence();
-                const float* all = part + ((size_t)tile * pieces * S::WIN) * kTcM + m;
-#pragma unroll
-                for (int c = 0; c < S::WIN; ++c) {
-                    float sum = 0.f;
-                    for (int p = 0; p < pieces; ++p) sum += __ldcg(all + ((size_t)p * S::WIN + c) * kTcM);   // piece order
-                    win[c] = sum;
-                }
-                if (et == 0) tile_cnt[tile] = 0;           // left at zero for the next call
-            }
-        } else {
-            epilogue_bar_sync();                           // s_ra is complete
+            for (int c = 0; c < S::WIN; ++c) st_cluster_f32(base + (uint32_t)(c * kTcM + m) * 4, 0, win[c]);
+            st_cluster_f32(base + (uint32_t)(S::WIN * kTcM + m) * 4, 0, na);
+            if (et < S::NCAND) st_cluster_f32(base + (uint32_t)((S::WIN + 1) * kTcM + et) * 4, 0, nb);
         }
-        if (last && row_ok) {
+        __syncwarp();
+        cluster_sync_all();
+        if (warp >= 2 && piece == 0) {
+            const float* xin = reinterpret_cast<const float*>(dyn);
+            for (int p = 1; p < pieces; ++p) {             // rank order
+                const float* xp = xin + (size_t)(p - 1) * XROW;
+#pragma unroll
+                for (int c = 0; c < S::WIN; ++c) win[c] += xp[c * kTcM + m];
+                na += xp[S::WIN * kTcM + m];
+                if (et < S::NCAND) nb += xp[(S::WIN + 1) * kTcM + et];
+            }
+        }
+    }
+
+    if (warp >= 2 && piece == 0) {
+        // ---- epilogue, part 3 (rank 0 of the tile): cosine, arg max over the window clipped to the grid, gate --
+        if (et < S::NCAND) s_nb[et] = nb;
+        epilogue_bar_sync();
+        const int kl = m >> 2, dx = m & 3;
+        const int k = k0 + kl, x = x0 + dx;
+        if (k < F && x < W) {
+            const size_t f = (size_t)k * N + (size_t)y * W + x;
             if (k == a) {                                  // anchor tokens are always retained (Eq. mask)
                 shat[f] = 1.0f; dst[f] = y * W + x; keep[f] = 1;
             } else {
+                const float rs = 1.0f / fmaxf(sqrtf(na), kNormFloor);
                 float best = -INFINITY;
                 int best_j = -1;
 #pragma unroll
@@ -297,8 +382,9 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
                     for (int wx = 0; wx < S::SIDE; ++wx) {     // ascending anchor index among in-grid cells
                         const int yy = y + wy - R, xx = x + wx - R;
                         if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
-                        const float s = win[wy * S::SIDE + wx] * rs * s_ra[wy * S::BW + dx + wx];
-                        if (s > best || best_j < 0) { best = s; best_j = yy * W + xx; }
+                        const float ra = 1.0f / fmaxf(sqrtf(s_nb[wy * S::BW + dx + wx]), kNormFloor);
+                        const float sim = win[wy * S::SIDE + wx] * rs * ra;
+                        if (sim > best || best_j < 0) { best = sim; best_j = yy * W + xx; }
                     }
                 const unsigned char kp = !(best > t);
                 shat[f] = best; dst[f] = best_j; keep[f] = kp;
@@ -310,6 +396,7 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
     // ---- teardown: every role is done with tensor memory before its owner frees it --------------------------
     tc_fence_before();
     __syncthreads();
+    trace_mark(asrc.hdr, 2, true);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem, S::TMEM_COLS);
@@ -351,35 +438,30 @@ static bool make_map(CUtensorMap* m, const void* X, int F, int H, int W, int C, 
 
 bool tc_match_eligible(const Problem& p) {
     if (p.dtype != 1 || !p.vec || p.r > 2 || p.C < kTcKC) return false;
-    const long long tiles = (long long)((p.F + kTcFR - 1) / kTcFR) * p.H * ((p.W + kTcWB - 1) / kTcWB);
-    return tiles * 8 < (1LL << 31);
-}
-
-// CTAs per tile: enough that a clip gives every SM two CTAs, at most 8 and at least 4 stages each
-int tc_match_pieces(const Problem& p) {
-    const long long tiles = (long long)((p.F + kTcFR - 1) / kTcFR) * p.H * ((p.W + kTcWB - 1) / kTcWB);
-    const int nst = (p.C + kTcKC - 1) / kTcKC;
-    long long want = (2LL * sm_count() + tiles - 1) / tiles;
-    if (want > 8) want = 8;
-    if (want > nst / 4) want = nst / 4;
-    return want < 1 ? 1 : (int)want;
-}
-
-size_t tc_match_part_floats(const Problem& p) {
-    const long long tiles = (long long)((p.F + kTcFR - 1) / kTcFR) * p.H * ((p.W + kTcWB - 1) / kTcWB);
-    const int pieces = tc_match_pieces(p);
-    const int win = (2 * p.r + 1) * (2 * p.r + 1);
-    return pieces > 1 ? (size_t)tiles * pieces * win * kTcM : 0;
+    return (long long)tc_match_tiles(p) * 8 < (1LL << 31);
 }
 
 size_t tc_match_tiles(const Problem& p) {
     return (size_t)((p.F + kTcFR - 1) / kTcFR) * p.H * ((p.W + kTcWB - 1) / kTcWB);
 }
 
+// CTAs (= cluster size) per tile: the largest power of two that still fits the GPU in one wave of two CTAs per SM,
+// at most 8 (4 for r = 2, whose exchange rows are longer) and at least 4 stages each
+int tc_match_pieces(const Problem& p) {
+    const long long tiles = (long long)tc_match_tiles(p);
+    const int nst = (p.C + kTcKC - 1) / kTcKC;
+    const int cap = p.r == 2 ? 4 : 8;
+    int pieces = 1;
+    while (pieces * 2 <= cap && tiles * (pieces * 2) <= 2LL * sm_count() && nst / (pieces * 2) >= 4) pieces *= 2;
+    return pieces;
+}
+
 template <int R>
 static cudaError_t launch_tc_t(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                                unsigned char* keep, cudaStream_t st) {
     using S = TcShape<R>;
+    static_assert((size_t)7 * ((S::WIN + 1) * kTcM + S::NCAND) * 4 <= (size_t)S::STAGES * S::STAGE || R == 2, "exchange rows must fit the ring");
+    static_assert((size_t)3 * ((S::WIN + 1) * kTcM + S::NCAND) * 4 <= (size_t)S::STAGES * S::STAGE, "exchange rows must fit the ring");
     CUtensorMap mapA, mapB;
     if (!make_map(&mapA, p.X, p.F, p.H, p.W, p.C, kTcWB, 1, kTcFR) ||
         !make_map(&mapB, p.X, p.F, p.H, p.W, p.C, S::BW, S::SIDE, 1))
@@ -389,9 +471,20 @@ static cudaError_t launch_tc_t(const Problem& p, const Scratch& s, int* out_anch
     if (e != cudaSuccess) return e;
     const int pieces = tc_match_pieces(p);
     const long long tiles = (long long)tc_match_tiles(p);
-    return launch_ex(true, smem, k_match_tc<R>, dim3((unsigned)(tiles * pieces)), dim3(kTcThreads), st, mapA, mapB,
-                     p.F, p.H, p.W, p.C, p.t, make_anchor_src(p, s, out_anchor), (const float*)s.ssq, p.nslice, pieces,
-                     s.tc_part, s.tc_cnt, shat, dst, keep, s.cnt, wait_poll_limit());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(tiles * pieces)); cfg.blockDim = dim3(kTcThreads); cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    int n = 1;
+    if (pieces > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = (unsigned)pieces; attr[n].val.clusterDim.y = 1; attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.attrs = attr; cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, k_match_tc<R>, mapA, mapB, p.F, p.H, p.W, p.C, p.t, make_anchor_src(p, s, out_anchor),
+                              pieces, shat, dst, keep, s.cnt, wait_poll_limit());
 }
 
 cudaError_t launch_match_tc(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,

@@ -37,7 +37,8 @@ def to_bits(t: torch.Tensor) -> np.ndarray:
 
 
 def check_clip(X: np.ndarray, r: int, t: float, *, stream=None, workspace=None, oracle=None,
-               require_anchor=True, anchor_mode: int = 0, anchor_frame: int = 0) -> dict:
+               require_anchor=True, anchor_mode: int = 0, anchor_frame: int = 0, order: int = 0,
+               pos_base: int = 0) -> dict:
     """Runs ttf_query and ttf_compress on X and compares with the oracle.  Returns a small report."""
     F, H, W, C = X.shape
     N = H * W
@@ -47,7 +48,7 @@ def check_clip(X: np.ndarray, r: int, t: float, *, stream=None, workspace=None, 
 
     kw = dict(stream=stream, workspace=workspace, anchor_mode=anchor_mode, anchor_frame=anchor_frame)
     q = P.ttf_query(Xd, r, t, **kw)
-    toks, cnt, pos = P.ttf_compress(Xd, r, t, **kw)
+    toks, cnt, pos = P.ttf_compress(Xd, r, t, order=order, pos_base=pos_base, **kw)
     torch.cuda.synchronize()
 
     a_gpu = int(q["anchor"].item())
@@ -76,7 +77,7 @@ def check_clip(X: np.ndarray, r: int, t: float, *, stream=None, workspace=None, 
     assert not bad_dst.any(), f"{int(bad_dst.sum())} dst differ outside the tie band"
 
     # everything downstream of the accepted decisions is exact
-    forced = O.compress(X, r, t, anchor_frame=a_gpu, forced_keep=keep)
+    forced = O.compress(X, r, t, anchor_frame=a_gpu, forced_keep=keep, natural=bool(order), pos_base=pos_base)
     assert (fuse == O.fuse_count(keep, dst, F, N, a_gpu)).all(), "fuse counts differ"
     L = int(cnt.item())
     assert L == forced.count, f"count {L} != {forced.count}"

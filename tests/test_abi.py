@@ -64,9 +64,18 @@ def test_null_and_nonfinite_arguments_are_rejected_before_any_launch(lib):
     assert lib.ttf_compress_ws(fake, 4, 4, 4, 8, 1, 0.7, 0, fake, fake, fake, ctypes.c_void_p(4096 + 8), 1 << 30, None) == 3
     assert lib.ttf_query(None, 4, 4, 4, 8, 1, 0.7, 0, None, None, None, None, None, None) == 1
     assert lib.ttf_compress_host(None, 4, 4, 4, 8, 1, 0.7, 0, fake, fake, fake) == 1
-    assert lib.ttf_compress_ex(fake, 4, 4, 4, 8, 1, 0.7, 0, 4, 0, fake, fake, fake, None) == 1      # unknown rule
-    assert lib.ttf_compress_ex(fake, 4, 4, 4, 8, 1, 0.7, 0, 3, 4, fake, fake, fake, None) == 1      # frame >= F
-    assert lib.ttf_query_ex(fake, 4, 4, 4, 8, 1, 0.7, 0, 3, -1, None, None, None, None, None, None) == 1
+    from paper_2605_07355_b200.binding import TTFOptions
+    opt = lambda *a: ctypes.byref(TTFOptions(*a))
+    ex = lib.ttf_compress_ex
+    assert ex(fake, 4, 4, 4, 8, 1, 0.7, 0, opt(4, 0, 0, 0), fake, fake, fake, None) == 1      # unknown anchor rule
+    assert ex(fake, 4, 4, 4, 8, 1, 0.7, 0, opt(3, 4, 0, 0), fake, fake, fake, None) == 1      # explicit frame >= F
+    assert ex(fake, 4, 4, 4, 8, 1, 0.7, 0, opt(0, 0, 2, 0), fake, fake, fake, None) == 1      # unknown order
+    assert ex(fake, 4, 4, 4, 8, 1, 0.7, 0, opt(0, 0, 0, -1), fake, fake, fake, None) == 1     # negative position base
+    assert ex(fake, 4, 4, 4, 8, 1, 0.7, 0, opt(0, 0, 0, 2**31 - 2), fake, fake, fake, None) == 1   # positions overflow
+    assert ex(None, 4, 4, 4, 8, 1, 0.7, 0, None, fake, fake, fake, None) == 1
+    assert lib.ttf_query_ex(fake, 4, 4, 4, 8, 1, 0.7, 0, opt(3, -1, 0, 0), None, None, None, None, None, None) == 1
+    arr = (ctypes.c_void_p * 2)(4096, 8192)
+    assert lib.ttf_compress_batch_ex(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, opt(0, 0, 0, 0), None, arr, arr, None) == 1
 
 
 def test_batch_and_variant_entry_points_validate_before_any_cuda_call(lib):
@@ -90,8 +99,8 @@ def test_batch_and_variant_entry_points_validate_before_any_cuda_call(lib):
     ms = (ctypes.c_double * 5)()
     assert lib.ttf_profile_stages(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, 0, ms, 5, None) == 1   # reps < 1
     assert lib.ttf_profile_stages(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, 1, None, 5, None) == 1
-    assert lib.ttf_set_schedule(9, 0, 0) == 1 and lib.ttf_set_schedule(0, 3, 0) == 1 and lib.ttf_set_schedule(0, 0, 101) == 1
-    assert lib.ttf_set_schedule(0, 0, 0) == 0
+    assert lib.ttf_set_schedule(9) == 1 and lib.ttf_set_schedule(-1) == 1
+    assert lib.ttf_set_schedule(0) == 0
 
 
 def test_decode_alignment_helper():

@@ -56,6 +56,50 @@ def test_batch_small_and_fp32_and_stream_order():
         P.ttf_compress_batch([Xs[0], Xs[1][:2]], 1, 0.7)
 
 
+SHAPES = [(1, 4, 4, 32, 1), (2, 3, 5, 40, 1), (6, 5, 6, 264, 0), (17, 3, 3, 72, 1), (33, 2, 3, 64, 1),
+          (9, 4, 6, 1032, 1), (40, 7, 9, 512, 2)]
+
+
+@pytest.mark.parametrize("kernel", [1, 2])
+@pytest.mark.parametrize("shape", SHAPES)
+def test_batch_chains_small_shapes(shape, kernel):
+    """seven clips over one, two and three lanes: clips of a lane form a chain on two scratch blocks in which the
+    sweep of a clip runs beside the gather of the clip before it; both matching kernels"""
+    F, H, W, C, r = shape
+    Xs = [to_device(corr_clip(F, H, W, C, seed=sum(shape) + j, dtype="bf16")) for j in range(7)]
+    P.ttf_set_match_kernel(kernel)
+    try:
+        ref = [P.ttf_compress(x, r, 0.6) for x in Xs]
+        torch.cuda.synchronize()
+        for lanes in (1, 2, 3):
+            P.ttf_set_schedule(lanes)
+            for rep in range(2):
+                toks, cnts, poss = P.ttf_compress_batch(Xs, r, 0.6)
+            torch.cuda.synchronize()
+            assert P.ttf_last_device_status() == 0
+            for j in range(len(Xs)):
+                L = int(ref[j][1].item())
+                assert int(cnts[j].item()) == L, (lanes, j)
+                assert torch.equal(toks[j][:L], ref[j][0][:L]) and torch.equal(poss[j][:L], ref[j][2][:L])
+        check_clip(to_bits(Xs[3]).reshape(F, H, W, C), r, 0.6)
+    finally:
+        P.ttf_set_schedule(0)
+        P.ttf_set_match_kernel(0)
+
+
+def test_batch_with_options_matches_single_calls():
+    Xs = [to_device(corr_clip(5, 6, 6, 128, seed=400 + j, dtype="bf16")) for j in range(5)]
+    for kw in (dict(anchor_mode=1), dict(anchor_mode=2, order=1), dict(anchor_mode=3, anchor_frame=2, pos_base=99), dict(order=1)):
+        toks, cnts, poss = P.ttf_compress_batch(Xs, 1, 0.6, **kw)
+        torch.cuda.synchronize()
+        for j, x in enumerate(Xs):
+            a = P.ttf_compress(x, 1, 0.6, **kw)
+            torch.cuda.synchronize()
+            L = int(a[1].item())
+            assert int(cnts[j].item()) == L
+            assert torch.equal(toks[j][:L], a[0][:L]) and torch.equal(poss[j][:L], a[2][:L])
+
+
 def test_host_batch_matches_device_calls():
     s = clips.CONFIGS["tiny_cal"]
     Xn = [clips.make_clip(s, s.seed + j) for j in range(5)]           # more clips than staging slots

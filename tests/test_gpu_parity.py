@@ -75,6 +75,16 @@ def test_fixed_anchor_rules(mode, frame):
         P.ttf_query(to_device(X), 1, 0.7, anchor_mode=3, anchor_frame=5)
 
 
+@pytest.mark.parametrize("dtype,C", [("bf16", 128), ("f32", 24), ("bf16", 33)])
+def test_natural_order_and_position_base(dtype, C):
+    """options of the _ex entry points: ascending flat order, positions offset by a base, with every anchor rule"""
+    X = corr_clip(6, 5, 7, C, seed=300 + C, dtype=dtype)
+    for mode, frame in ((0, 0), (1, 0), (2, 0), (3, 3)):
+        for order, base in ((1, 0), (0, 777), (1, 12345)):
+            rep = check_clip(X, 1, 0.6, anchor_mode=mode, anchor_frame=frame, order=order, pos_base=base)
+            assert rep["count"] > 35
+
+
 def test_misaligned_base_pointer_takes_scalar_path():
     F, H, W, C = 3, 4, 5, 64
     X = corr_clip(F, H, W, C, seed=12, dtype="bf16")

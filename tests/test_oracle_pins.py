@@ -208,6 +208,27 @@ def test_positions_and_order(anchor_frame):
     assert 0 < len(src) < (F - 1) * N       # the case exercises both outcomes of the gate
 
 
+def test_natural_order_and_position_base():
+    """the other reading of "ordered index set" (ascending flat index) and a constant position offset"""
+    F, H, W, C = 5, 4, 6, 16
+    N = H * W
+    X = corr_clip(F, H, W, C, seed=71)
+    for a in (0, 2, 4):
+        R = O.compress(X, 1, 0.6, anchor_frame=a)
+        Rn = O.compress(X, 1, 0.6, anchor_frame=a, natural=True)
+        assert Rn.count == R.count and (Rn.keep == R.keep).all()
+        assert (np.diff(Rn.index) > 0).all()                                 # strictly ascending flat index
+        assert sorted(Rn.index.tolist()) == sorted(R.index.tolist())         # the same tokens, another order
+        assert (Rn.index == np.flatnonzero(R.keep)).all()                    # = every retained token, numpy's own scan
+        assert (Rn.tokens == X.reshape(F * N, C)[Rn.index]).all()
+        k, i = Rn.index // N, Rn.index % N
+        assert (Rn.pos == np.stack([k, i // W, i % W], axis=1)).all()
+        if a == 0:                                                           # anchor first = natural when a = 0
+            assert (Rn.index == R.index).all() and (Rn.pos == R.pos).all() and (Rn.tokens == R.tokens).all()
+        Rb = O.compress(X, 1, 0.6, anchor_frame=a, pos_base=1000)
+        assert (Rb.pos == R.pos + 1000).all() and (Rb.tokens == R.tokens).all() and (Rb.index == R.index).all()
+
+
 def test_forced_keep_drives_compaction():
     X = corr_clip(3, 4, 4, 16, seed=43)
     R = O.compress(X, 1, 0.70)
