@@ -41,8 +41,11 @@ def parse_args():
     ap.add_argument("--workload", default="vl8b_cal")
     ap.add_argument("--clips", type=int, default=16, help="distinct clips per step (batch)")
     ap.add_argument("--streams", type=int, default=0,
-                    help="0: one ttf_compress_batch call per step (the library spreads the clips over its own four "
-                         "streams); S > 0: one ttf_compress call per clip on S streams of the caller")
+                    help="0: one ttf_compress_batch call per step (the library spreads the clips over its own "
+                         "streams, see --lanes); S > 0: one ttf_compress call per clip on S streams of the caller")
+    ap.add_argument("--lanes", type=int, default=0, help="clips of a batch in flight (ttf_set_schedule); 0 = automatic")
+    ap.add_argument("--match-kernel", default="auto", choices=["auto", "mma", "tc"],
+                    help="kernel of the matching step for bf16 clips (ttf_set_match_kernel)")
     ap.add_argument("--threshold", type=float, default=None)
     ap.add_argument("--anchor", default="auto", choices=["auto", "first", "last"], help="anchor rule")
     ap.add_argument("--no-graph", action="store_true",
@@ -54,10 +57,20 @@ def parse_args():
     return ap.parse_args()
 
 
-# DRAM bytes (read + write) per launch from the committed ncu capture (profiles/kernels_full_vl8b_cal.md: cold
-# caches, one launch of each kernel).  Valid only for the kernels as captured; other workloads report null.
-NCU_TRAFFIC = {("vl8b_cal", "match"): 67141888 + 1333248, ("vl8b_cal", "norm_sum"): 67120128 + 563968,
-               ("vl8b_cal", "compact"): 24693760 + 80896}
+def stored_traffic(workload: str, kernel: str, csrc: str):
+    """DRAM bytes (read + write) per launch of `kernel` from the stored profiler counters, or None when there are
+    none for this workload or they were taken on other sources than the library was built from."""
+    path = os.path.join(ROOT, "profiles", f"dram_per_kernel_{workload}.json")
+    try:
+        d = json.load(open(path))
+    except Exception:
+        return None, "no stored counters for this workload"
+    if d.get("csrc_hash") != csrc:
+        return None, "stored counters were taken on other kernel sources"
+    k = d.get("kernels", {}).get(kernel)
+    if not k:
+        return None, "no stored counters for this kernel"
+    return int(k["dram_bytes_read"]) + int(k["dram_bytes_write"]), d.get("note", "ncu, one launch")
 
 
 def peaks():
@@ -216,10 +229,10 @@ def combine_ranks(ms_local: float, tokens_local: int, device=None):
     return float(t.item()), int(n.item())
 
 
-def workload_config(spec, t, clips_per_step, streams, tokens_per_step, anchor="auto", graph=False):
+def workload_config(spec, t, clips_per_step, streams, tokens_per_step, anchor="auto", graph=False, match_kernel="auto"):
     return {"workload": f"{spec.name}: F={spec.F} {spec.H}x{spec.W} C={spec.C} {spec.dtype} r={spec.r} t={t:.2f}",
             "generator": spec.family, "clips_per_step": clips_per_step, "tokens_per_step": tokens_per_step,
-            "streams": streams, "anchor": anchor, "cuda_graph": graph,
+            "streams": streams, "anchor": anchor, "cuda_graph": graph, "match_kernel": match_kernel,
             "l2": "inputs rotate through a batch larger than L2; every clip starts cold in HBM"}
 
 
@@ -278,12 +291,13 @@ def main():
     joins = [torch.cuda.Event() for _ in streams]
 
     amode = {"auto": 0, "first": 1, "last": 2}[args.anchor]
-    if args.streams == 0 and amode != 0:
-        raise SystemExit("--anchor first/last needs --streams S > 0 (ttf_compress_batch uses the automatic anchor)")
+    P.ttf_set_match_kernel({"auto": 0, "mma": 1, "tc": 2}[args.match_kernel])
+    P.ttf_set_schedule(args.lanes)
+    lanes = args.lanes if args.lanes > 0 else 8
 
     def step():
         if args.streams == 0:
-            P.ttf_compress_batch(devX, spec.r, t, out_tok, out_cnt, out_pos, stream=main_stream)
+            P.ttf_compress_batch(devX, spec.r, t, out_tok, out_cnt, out_pos, stream=main_stream, anchor_mode=amode)
             return
         if nstreams == 1:
             for j in range(nclips):
@@ -331,21 +345,44 @@ def main():
     sampler.start()
     time.sleep(0.05)
 
-    # ---- timed region: exactly K steps, CUDA events on the launching stream -------------------------------
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # ---- timed region: exactly K steps, CUDA events on the launching stream (one event after every step, so
+    # that the spread over the steps is known as well as the total) ------------------------------------------
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
     w0 = time.perf_counter()
-    e0.record(main_stream)
-    for _ in range(args.steps):
+    marks[0].record(main_stream)
+    for i in range(args.steps):
         step()
-    e1.record(main_stream)
+        marks[i + 1].record(main_stream)
     barrier()
     w1 = time.perf_counter()
     tokens_step = nclips * FN
-    ms_total, tokens_all = combine_ranks(e0.elapsed_time(e1), tokens_step, dev)
+    ms_total, tokens_all = combine_ranks(marks[0].elapsed_time(marks[-1]), tokens_step, dev)
     ms_step = ms_total / args.steps
     value = tokens_all / (ms_step * 1e-3)
     clips_per_s = value / FN
+    per_step = sorted(marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps))
+    pick = lambda q: per_step[min(len(per_step) - 1, int(q * len(per_step)))]
+    step_ms = {"median": pick(0.5), "p10": pick(0.1), "p90": pick(0.9), "min": per_step[0], "max": per_step[-1]}
+
+    # ---- latency of one clip when nothing else is in flight: the clips of the step one after the other on one
+    # stream (captured like the step itself) ------------------------------------------------------------------
+    lat_graph = torch.cuda.CUDAGraph()
+    for j in range(min(nclips, 4)):
+        P.ttf_compress(devX[j], spec.r, t, out_tok[j], out_cnt[j], out_pos[j], stream=main_stream, anchor_mode=amode)
+    barrier()
+    with torch.cuda.graph(lat_graph, stream=main_stream):
+        for j in range(nclips):
+            P.ttf_compress(devX[j], spec.r, t, out_tok[j], out_cnt[j], out_pos[j], stream=main_stream, anchor_mode=amode)
+    l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(main_stream):
+        lat_graph.replay()
+        l0.record(main_stream)
+        for _ in range(5):
+            lat_graph.replay()
+        l1.record(main_stream)
+    barrier()
+    latency_us = l0.elapsed_time(l1) * 1e3 / (5 * nclips)
 
     # ---- per-kernel durations at steady state: every kernel launched back to back for all clips of the step,
     # CUDA events (on the launching stream) around each group, divided by the clips; the batch is larger than L2,
@@ -355,7 +392,9 @@ def main():
     kernel_ms = P.ttf_profile_stages(devX, spec.r, t, out_tok, out_cnt, out_pos, reps=min(args.steps, 20),
                                      stream=main_stream)
     torch.cuda.synchronize()
-    launches_per_step = 4 * nclips if amode == 0 else 3 * nclips
+    launches_per_step = 4 * nclips      # sweep (or its stand-in for a fixed anchor), statistics or none, matching, gather
+    if amode != 0:
+        launches_per_step = 3 * nclips
     kern = {k: {"us_per_launch": 1e3 * v} for k, v in kernel_ms.items() if v > 0}
     tot = sum(kernel_ms.values())
     dominant = max(kern, key=lambda k: kernel_ms[k])
@@ -363,12 +402,13 @@ def main():
     avg_count = sum(counts) / nclips
     kbytes = A.kernel_bytes(dominant, spec.F, spec.N, C, spec.itemsize, int(round(avg_count)))
     achieved = kbytes / (kern[dominant]["us_per_launch"] * 1e-6) / 1e9
+    csrc = A.csrc_hash()
+    traffic, traffic_note = stored_traffic(spec.name, dominant, csrc) if amode == 0 else (None, "no stored counters for this anchor rule")
     roofline = {"bound": "hbm", "kernel": dominant,
                 "timed": "each kernel launched back to back for the clips of a step (cold in HBM), CUDA events around the group, / clips",
                 "achieved": achieved, "peak": peak_gbs, "unit": "GB/s",
                 "frac": achieved / peak_gbs, "peak_source": f"of {peak_kind}",
-                "traffic": NCU_TRAFFIC.get((spec.name, dominant)) if amode == 0 else None,
-                "traffic_note": "ncu, cold caches, one launch",
+                "traffic": traffic, "traffic_note": traffic_note, "csrc_hash": csrc,
                 "algorithmic_bytes_per_launch": kbytes,
                 "kernel_share": {k: kernel_ms[k] / tot for k in kern},
                 "kernel_us": {k: round(kern[k]["us_per_launch"], 3) for k in kern},
@@ -376,8 +416,13 @@ def main():
                                 / (kern[k]["us_per_launch"] * 1e-6) / 1e9 / peak_gbs for k in kern}}
     bmin = A.pass_bytes(spec.F, spec.N, C, spec.itemsize, int(round(avg_count)))
     pass_gbs = bmin * nclips / (ms_step * 1e-3) / 1e9
+    model = A.pipeline_dram_bytes_model(spec.F, spec.N, C, spec.itemsize, int(round(avg_count)),
+                                        lanes if args.streams == 0 else nstreams)
     pass_roofline = {"bytes_per_clip": bmin, "achieved": pass_gbs, "unit": "GB/s", "frac_of_measured_copy": pass_gbs / peak_gbs,
-                     "frac_of_8TBps": pass_gbs / 8000.0, "us_per_clip": ms_step * 1e3 / nclips}
+                     "frac_of_8TBps": pass_gbs / 8000.0, "us_per_clip": ms_step * 1e3 / nclips,
+                     "dram_bytes_per_clip_model": model,
+                     "model_frac_of_measured_copy": model * nclips / (ms_step * 1e-3) / 1e9 / peak_gbs,
+                     "latency_us_per_clip_one_stream": latency_us}
 
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region --------------------
     e2e = None
@@ -413,9 +458,10 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": workload_config(spec, t, nclips, "8 (library: ttf_compress_batch)" if args.streams == 0 else nstreams,
-                                      tokens_step, args.anchor, use_graph),
+            "vs_baseline": None, "dtype": spec.dtype, "accumulate": "f32", "data": "synthetic",
+            "config": workload_config(spec, t, nclips, f"{lanes} (library: ttf_compress_batch)" if args.streams == 0 else nstreams,
+                                      tokens_step, args.anchor, use_graph, args.match_kernel),
+            "step_ms": step_ms,
             "clips_per_s": clips_per_s, "rho": rho, "count_mean": avg_count,
             "roofline": roofline, "pass_roofline": pass_roofline, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": int(launches_per_step * args.steps), "gpu_launches_per_step": int(launches_per_step),

@@ -40,3 +40,32 @@ def kernel_bytes(kind: str, F: int, N: int, C: int, itemsize: int, count: int) -
     if kind == "compact":           # reads the retained rows, writes them with their positions
         return 2 * count * C * itemsize + count * 12 + F * N + 4
     raise KeyError(kind)
+
+
+def pipeline_dram_bytes_model(F: int, N: int, C: int, itemsize: int, count: int, lanes: int) -> int:
+    """DRAM bytes one clip moves in the pipeline as scheduled.  With one clip in flight the matching pass and the
+    gather find the clip in L2 (measured: about 3 MB and 1 MB of DRAM reads), so the clip is read once; with
+    several clips in flight they displace one another, and the second pass over X and the gather's rows come from
+    DRAM again.  Output rows, positions and the small per-token arrays are written once either way."""
+    X = F * N * C * itemsize
+    rows = count * C * itemsize
+    small = F * N * 9 + count * 12 + 4
+    if lanes <= 1:
+        return X + rows + small
+    return 2 * X + 2 * rows + small
+
+
+def csrc_hash() -> str:
+    """Hash of the CUDA sources and the C header the library is built from: ties stored profiler counters to the
+    kernels they were taken on."""
+    import glob
+    import hashlib
+    import os
+    here = os.path.dirname(os.path.abspath(__file__))
+    files = sorted(glob.glob(os.path.join(here, "csrc", "*.cu")) + glob.glob(os.path.join(here, "csrc", "*.cuh")))
+    files.append(os.path.join(os.path.dirname(here), "include", "ttf.h"))
+    h = hashlib.sha256()
+    for f in files:
+        h.update(os.path.basename(f).encode())
+        h.update(open(f, "rb").read())
+    return h.hexdigest()[:16]

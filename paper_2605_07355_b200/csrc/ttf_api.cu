@@ -3,6 +3,8 @@
 #include "../../include/ttf.h"
 #include "ttf_internal.cuh"
 
+#include <nvtx3/nvToolsExt.h>
+
 #include <atomic>
 #include <cmath>
 #include <cstdlib>
@@ -75,9 +77,15 @@ static std::mutex g_prof_mu;
 static bool g_prof_on = false;
 static std::vector<ProfRecord> g_prof;
 
+static const char* const kKindNames[PK_KINDS] = {"ttf sweep", "ttf frame statistics", "ttf matching", "ttf gather",
+                                                 "ttf fuse count"};
+
+// One scope per kernel launch: an NVTX range on the host side of the launch (a no-op unless a tool that listens is
+// attached) and, while profiling is on, a pair of CUDA events around it.
 struct ProfScope {
     cudaStream_t st; int kind; cudaEvent_t a = nullptr, b = nullptr; bool on;
-    ProfScope(cudaStream_t s, int k) : st(s), kind(k), on(g_prof_on) {
+    struct Range { Range(int k) { nvtxRangePushA(kKindNames[k]); } ~Range() { nvtxRangePop(); } } range;
+    ProfScope(cudaStream_t s, int k) : st(s), kind(k), on(g_prof_on), range(k) {
         if (!on) return;
         if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { on = false; return; }
         cudaEventRecord(a, st);

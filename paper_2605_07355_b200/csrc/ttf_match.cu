@@ -131,14 +131,8 @@ k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, flo
 // r = 2: the 25 candidate rows of a cell are as much data as 25 source rows, so a CTA takes 64 frames per cell to
 // amortise them (2.6 -> 1.4 times |X| of operand traffic); norms come from the sweep, which frees the registers
 // of the Gram accumulators for the 64 x 32 tile of dot products.
-#ifndef TTF_WIDE_MT
-#define TTF_WIDE_MT 4
-#endif
-#ifndef TTF_WIDE_STAGES
-#define TTF_WIDE_STAGES 2
-#endif
-constexpr int kWideMT = TTF_WIDE_MT;
-constexpr int kWideStages = TTF_WIDE_STAGES;
+constexpr int kWideMT = 4;           // 64 frames per CTA
+constexpr int kWideStages = 2;       // cp.async stages per warp (the 64 x 32 accumulator tile leaves no room for more)
 __global__ void __launch_bounds__(kMmaWarps * 32, 2)
 k_match_mma_wide(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t, AnchorSrc asrc,
                  const float* __restrict__ ssq, int nslice,

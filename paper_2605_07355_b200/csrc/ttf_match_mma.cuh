@@ -33,13 +33,8 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
 }
 
 constexpr int kMmaWarps = 8;
-#ifndef TTF_MMA_STAGES
-#define TTF_MMA_STAGES 3
-#endif
-#ifndef TTF_MMA_MAXREG
-#define TTF_MMA_MAXREG 96
-#endif
-constexpr int kMmaStagesDefault = TTF_MMA_STAGES; // cp.async stages per warp (stages - 1 blocks in flight)
+constexpr int kMmaStagesDefault = 3; // cp.async stages per warp (stages - 1 blocks in flight)
+constexpr int kMmaMaxReg = 96;       // registers per thread of the r <= 1 kernel (see TTF_MMA_BOUNDS)
 
 // One pipeline stage of a warp: the 16-byte fragment pieces of its 64-byte block, (2 MT + NT) per lane.  The
 // pieces travel global -> shared with cp.async (no registers are tied up while they are in flight, so a warp
@@ -111,7 +106,7 @@ __device__ __forceinline__ void mma_consume_stage(const uint4* slot, int lane, f
 
 // 96 registers and 3 stages (74 KB) per CTA: two of these CTAs leave room on an SM for a CTA of the next clip's
 // sweep, which is what lets clips on different streams overlap (measured: 31.6 vs 33.3 us per clip, 4 streams)
-#define TTF_MMA_BOUNDS __maxnreg__(TTF_MMA_MAXREG)
+#define TTF_MMA_BOUNDS __maxnreg__(kMmaMaxReg)
 // GRAM: token norms from Gram-diagonal MMAs (else from the sweep's partial squared norms); ST: cp.async stages.
 //
 // One unit of work: cell i, frames k0 .. k0 + 16 MT - 1.  Called by all threads of a CTA of kMmaWarps warps;
