@@ -50,6 +50,10 @@ def parse_args():
     ap.add_argument("--anchor", default="auto", choices=["auto", "first", "last"], help="anchor rule")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every kernel from the host each step instead of replaying a captured CUDA graph")
+    ap.add_argument("--ncu-range", action="store_true",
+                    help="profiling aid: after the warm-up run ONE step between cudaProfilerStart/Stop and exit without "
+                         "timing anything (for `ncu --replay-mode range`, which measures the overlapped kernels of the "
+                         "step as one workload)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -324,6 +328,14 @@ def main():
     for _ in range(max(3, args.warmup)):
         launch_step()
     barrier()
+    if args.ncu_range:
+        torch.cuda.cudart().cudaProfilerStart()
+        launch_step()
+        torch.cuda.synchronize()
+        torch.cuda.cudart().cudaProfilerStop()
+        print(json.dumps({"ncu_range": "one step", "workload": spec.name, "clips_per_step": nclips, "lanes": lanes,
+                          "counts": [int(c.item()) for c in out_cnt]}), flush=True)
+        return
     use_graph = not args.no_graph
     if use_graph:
         # The step is launch-bound on the host (four kernels per clip, a few microseconds each to launch), so it

@@ -148,10 +148,11 @@ int ttf_compress_batch(const void* const* features, int nclips, int F, int H, in
 
 /*
  * Kernel of the matching step for bf16 clips with r <= 2 and 16-byte aligned rows (the paper has no counterpart; the
- * results are the same within the stated tolerance): 0 automatic; 1 the warp-level tensor-core MMA kernel (one cell
- * x 32 frames per CTA, token norms from Gram-tile diagonals); 2 the tcgen05 kernel (strips of 4 cells x 32 frames as
- * TMA tiles, accumulators in tensor memory, token norms from the sweep; needs C >= 64).  Process-wide; takes effect
- * with the next call.
+ * results are the same within the stated tolerance): 0 automatic (the faster of the two as measured: the tcgen05
+ * kernel for r = 2 and for clips with at least about 300 tiles of 32 frames x 4 cells, else the warp-level kernel);
+ * 1 the warp-level tensor-core MMA kernel (one cell x 32 frames per CTA, token norms from Gram-tile diagonals); 2 the
+ * tcgen05 kernel (strips of 4 cells x 32 frames as TMA tiles, accumulators in tensor memory, token norms taken from
+ * the tiles in shared memory; needs C >= 64).  Process-wide; takes effect with the next call.
  */
 int ttf_set_match_kernel(int which);
 
