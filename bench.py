@@ -328,14 +328,6 @@ def main():
     for _ in range(max(3, args.warmup)):
         launch_step()
     barrier()
-    if args.ncu_range:
-        torch.cuda.cudart().cudaProfilerStart()
-        launch_step()
-        torch.cuda.synchronize()
-        torch.cuda.cudart().cudaProfilerStop()
-        print(json.dumps({"ncu_range": "one step", "workload": spec.name, "clips_per_step": nclips, "lanes": lanes,
-                          "counts": [int(c.item()) for c in out_cnt]}), flush=True)
-        return
     use_graph = not args.no_graph
     if use_graph:
         # The step is launch-bound on the host (four kernels per clip, a few microseconds each to launch), so it
@@ -350,6 +342,14 @@ def main():
         for _ in range(3):
             step()
         barrier()
+    if args.ncu_range:
+        torch.cuda.cudart().cudaProfilerStart()
+        step()
+        torch.cuda.synchronize()
+        torch.cuda.cudart().cudaProfilerStop()
+        print(json.dumps({"ncu_range": "one step", "workload": spec.name, "clips_per_step": nclips, "lanes": lanes,
+                          "cuda_graph": use_graph, "counts": [int(c.item()) for c in out_cnt]}), flush=True)
+        return
     counts = [int(c.item()) for c in out_cnt]
     rho = 1.0 - sum(counts) / float(nclips * FN)
 
@@ -429,7 +429,7 @@ def main():
     bmin = A.pass_bytes(spec.F, spec.N, C, spec.itemsize, int(round(avg_count)))
     pass_gbs = bmin * nclips / (ms_step * 1e-3) / 1e9
     model = A.pipeline_dram_bytes_model(spec.F, spec.N, C, spec.itemsize, int(round(avg_count)),
-                                        lanes if args.streams == 0 else nstreams)
+                                        lanes if args.streams == 0 else nstreams, fixed_anchor=amode != 0)
     pass_roofline = {"bytes_per_clip": bmin, "achieved": pass_gbs, "unit": "GB/s", "frac_of_measured_copy": pass_gbs / peak_gbs,
                      "frac_of_8TBps": pass_gbs / 8000.0, "us_per_clip": ms_step * 1e3 / nclips,
                      "dram_bytes_per_clip_model": model,

@@ -42,17 +42,19 @@ def kernel_bytes(kind: str, F: int, N: int, C: int, itemsize: int, count: int) -
     raise KeyError(kind)
 
 
-def pipeline_dram_bytes_model(F: int, N: int, C: int, itemsize: int, count: int, lanes: int) -> int:
-    """DRAM bytes one clip moves in the pipeline as scheduled.  With one clip in flight the matching pass and the
-    gather find the clip in L2 (measured: about 3 MB and 1 MB of DRAM reads), so the clip is read once; with
-    several clips in flight they displace one another, and the second pass over X and the gather's rows come from
-    DRAM again.  Output rows, positions and the small per-token arrays are written once either way."""
+def pipeline_dram_bytes_model(F: int, N: int, C: int, itemsize: int, count: int, lanes: int, fixed_anchor: bool = False) -> int:
+    """DRAM bytes one clip moves in the pipeline as scheduled (confirmed with the profiler's DRAM counters over a
+    whole step: 93.6 / 160.2 / 178.3 MB per 8B-shaped clip for 1 / 2 / 8 clips in flight, 113.7 MB with a fixed
+    anchor).  With one clip in flight the matching pass and the gather find the clip in L2, so it is read once; with
+    two or more in flight the clips displace one another, and the second pass over X (which only the automatic anchor
+    of Eq. auto_anchor needs) and the gather's rows come from DRAM again.  Output rows, positions and the small
+    per-token arrays are written once either way."""
     X = F * N * C * itemsize
     rows = count * C * itemsize
     small = F * N * 9 + count * 12 + 4
     if lanes <= 1:
         return X + rows + small
-    return 2 * X + 2 * rows + small
+    return (1 if fixed_anchor else 2) * X + 2 * rows + small
 
 
 def csrc_hash() -> str:
