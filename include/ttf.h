@@ -256,7 +256,7 @@ int ttf_sim_histogram(const float* best_sim, const int* anchor, int F, int H, in
  * The same pass for callers whose tensors live in HOST memory (all four pointers are host pointers; pinned
  * memory makes the copies asynchronous).  Copies features to the device, runs ttf_compress, copies L' and the
  * first L' rows of tokens and positions back, and returns after synchronising.  Device staging buffers are
- * cached per device and reused.  out_count_host receives L'.
+ * cached per device and reused; calls from several host threads are serialised.  out_count_host receives L'.
  */
 int ttf_compress_host(const void* features_host, int F, int H, int W, int C, int r, float t, int dtype,
                       void* out_tokens_host, int* out_count_host, int* out_pos_thw_host);

@@ -74,7 +74,7 @@ int wait_tx_extra() { return g_wait_tx_extra.load(); }
 enum { PK_NORM_SUM = 0, PK_FRAME_STATS = 1, PK_MATCH = 2, PK_COMPACT = 3, PK_FUSE_COUNT = 4, PK_KINDS = 5 };
 struct ProfRecord { int kind; cudaEvent_t a, b; };
 static std::mutex g_prof_mu;
-static bool g_prof_on = false;
+static std::atomic<bool> g_prof_on{false};
 static std::vector<ProfRecord> g_prof;
 
 static const char* const kKindNames[PK_KINDS] = {"ttf sweep", "ttf frame statistics", "ttf matching", "ttf gather",
@@ -743,6 +743,10 @@ int ttf_compress_host(const void* features_host, int F, int H, int W, int C, int
     const size_t FN = (size_t)p.F * p.N;
     const size_t row_bytes = (size_t)C * esize;
 
+    // one host call at a time per process: the staging buffers and their stream are shared, and a second call with a
+    // larger clip would free buffers the first still uses
+    static std::mutex host_call_mu;
+    std::lock_guard<std::mutex> whole_call(host_call_mu);
     std::unique_lock<std::mutex> lk(g_mu);
     Staging& sg = g_staging[dev];
     if (!sg.stream) {

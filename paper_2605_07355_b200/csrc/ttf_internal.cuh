@@ -28,7 +28,7 @@ struct Problem {
     int N;              // H * W
     int vec;            // 1 when rows are 16-byte aligned and a multiple of 16 bytes long, else 0
     int lanes_elems;    // channels one lane loads at once: 16 B worth when vec, else 1
-    int ls;             // norm sweep: lanes across a channel slice (64, or 32 when that gives too few CTAs)
+    int ls;             // norm sweep: lanes across a channel slice (32: one warp)
     int nq;             // norm sweep: channel slices per row, ceil(C / (ls * lanes_elems))
     int nslice;         // planes of partial squared norms: one per warp across a slice, nq * ls / 32
     int nsl;            // frame statistics: channel slices (128 channels when C % 4 == 0, else 32)

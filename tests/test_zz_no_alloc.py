@@ -56,6 +56,25 @@ def test_static_scratch_query_matches_query_twice_in_a_row():
         assert torch.equal(a[k], b[k]), k
 
 
+def test_static_scratch_query_takes_no_device_memory():
+    """what the entry point exists for: once the address of the built-in array has been looked up, further calls
+    (another shape, another stream) leave the device's free memory exactly as it was"""
+    s0, s1 = clips.CONFIGS["tiny"], clips.CONFIGS["vl2b_cal"]
+    X0, X1 = to_device(clips.make_clip(s0)), to_device(clips.make_clip(s1))
+    out0, out1 = _outputs(s0.F, s0.N, -7), _outputs(s1.F, s1.N, -8)
+    st = torch.cuda.Stream()
+    P.ttf_query_static(X0, s0.r, s0.t, out0)                   # the first call on the device: address look-up
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    P.ttf_query_static(X1, s1.r, s1.t, out1)                   # a new shape ...
+    torch.cuda.synchronize()
+    P.ttf_query_static(X0, s0.r, s0.t, out0, stream=st)        # ... and a stream the library has never seen
+    st.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    _same(out1, P.ttf_query(X1, s1.r, s1.t))
+
+
 def test_static_scratch_limit_is_enforced_before_any_launch():
     lib = P.lib()
     fake = ctypes.c_void_p(4096)            # never dereferenced: the size check comes first
