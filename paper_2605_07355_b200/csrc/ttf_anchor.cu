@@ -285,8 +285,9 @@ k_frame_stats(const float* S, int F, int C, int nsl, float* Dp, float* Qp, float
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// The same statistics as ONE thread-block cluster of 8 CTAs, for clips whose frame sums fit its registers
-// (C <= 4096 channels and 32 / 64 / 128 frames for 4 / 2 / 1 slices of 128 channels per CTA).  A grid of
+// The same statistics as ONE thread-block cluster of 8 CTAs, for clips of at most 4096 channels and 256 frames (the
+// frame sums of 32 / 64 / 128 frames at 4 / 2 / 1 slices of 128 channels per CTA stay in registers; longer clips are
+// fetched a second time for the second step).  A grid of
 // independent CTAs has to go through global memory, a fence and an arrival counter before one of them can take
 // the arg max, which is five to six dependent round trips after the sweep; here every CTA fetches all of its
 // frame sums in one round trip, the per-frame shares of <S_k, g>, |S_k|^2 and |g|^2 go to rank 0 through
@@ -312,15 +313,17 @@ __device__ __forceinline__ void stat_st_cluster(const float* local, uint32_t ran
     asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
 }
 
-template <int SL>     // slices of 128 channels per CTA; FB = 16 / SL frames per thread (warp w owns frames w, w + 8, ...)
+constexpr int kStatClusterMaxF = 256;     // frames the cluster kernel takes (shares of all frames live in shared memory)
+
+template <int SL>     // slices of 128 channels per CTA; FB = 16 / SL frames per thread and chunk (warp w owns frames w, w + 8, ...)
 __global__ void __launch_bounds__(kNormThreads)
 k_frame_stats_cluster(const float* S, int F, int C, int nsl, int* hdr, int* out_anchor)
 {
     constexpr int FB = 16 / SL;
-    constexpr int MAXF = kNormWarps * FB;
+    constexpr int CHUNK = kNormWarps * FB;           // frames per chunk: 32 / 64 / 128
     __shared__ float4 s_g[SL][kNormWarps][32];
-    __shared__ float s_D[MAXF], s_Q[MAXF], s_G;
-    __shared__ float s_x[kStatCluster - 1][2 * MAXF + 1];      // what the other ranks send (rank 0 only)
+    __shared__ float s_D[kStatClusterMaxF], s_Q[kStatClusterMaxF], s_G;
+    __shared__ float s_x[kStatCluster - 1][2 * kStatClusterMaxF + 1];      // what the other ranks send (rank 0 only)
     __shared__ float s_best[kNormWarps];
     __shared__ int s_idx[kNormWarps];
     pdl_launch_dependents();
@@ -329,29 +332,40 @@ k_frame_stats_cluster(const float* S, int F, int C, int nsl, int* hdr, int* out_
     trace_mark(hdr, 4, false);
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
     const int rank = (int)stat_cluster_rank();
+    const bool one_chunk = F <= CHUNK;               // then the frame sums stay in registers for the second step
 
-    // one round trip: every frame sum this thread needs
+    // the frame sums of one chunk of frames: one round trip
     float4 v[SL][FB];
+    auto load_chunk = [&](int k0) {
 #pragma unroll
-    for (int sl = 0; sl < SL; ++sl) {
-        const int q = rank + sl * kStatCluster;
-        const int c0 = (q * 32 + lane) * 4;
+        for (int sl = 0; sl < SL; ++sl) {
+            const int q = rank + sl * kStatCluster;
+            const int c0 = (q * 32 + lane) * 4;
 #pragma unroll
-        for (int jj = 0; jj < FB; ++jj) {
-            const int kk = w + jj * kNormWarps;
-            v[sl][jj] = (q < nsl && c0 < C && kk < F) ? __ldcg(reinterpret_cast<const float4*>(S + (size_t)kk * C + c0))
-                                                      : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int jj = 0; jj < FB; ++jj) {
+                const int kk = k0 + w + jj * kNormWarps;
+                v[sl][jj] = (q < nsl && c0 < C && kk < F) ? __ldcg(reinterpret_cast<const float4*>(S + (size_t)kk * C + c0))
+                                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
         }
+    };
+    // step 1: g[c] = sum_k S_k[c] over all frames (chunks in order, then the warps in warp order)
+    float4 gacc[SL];
+#pragma unroll
+    for (int sl = 0; sl < SL; ++sl) gacc[sl] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k0 = 0; k0 < F; k0 += CHUNK) {
+        load_chunk(k0);
+#pragma unroll
+        for (int sl = 0; sl < SL; ++sl)
+#pragma unroll
+            for (int jj = 0; jj < FB; ++jj) {
+                gacc[sl].x += v[sl][jj].x; gacc[sl].y += v[sl][jj].y; gacc[sl].z += v[sl][jj].z; gacc[sl].w += v[sl][jj].w;
+            }
     }
 #pragma unroll
-    for (int sl = 0; sl < SL; ++sl) {
-        float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int jj = 0; jj < FB; ++jj) { g.x += v[sl][jj].x; g.y += v[sl][jj].y; g.z += v[sl][jj].z; g.w += v[sl][jj].w; }
-        s_g[sl][w][lane] = g;
-    }
+    for (int sl = 0; sl < SL; ++sl) s_g[sl][w][lane] = gacc[sl];
     __syncthreads();
-    float4 gl[SL];                                   // g[c] = sum_k S_k[c], warps combined in warp order
+    float4 gl[SL];
 #pragma unroll
     for (int sl = 0; sl < SL; ++sl) {
         float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -359,19 +373,23 @@ k_frame_stats_cluster(const float* S, int F, int C, int nsl, int* hdr, int* out_
         for (int ww = 0; ww < kNormWarps; ++ww) { const float4 t = s_g[sl][ww][lane]; g.x += t.x; g.y += t.y; g.z += t.z; g.w += t.w; }
         gl[sl] = g;
     }
+    // step 2: this CTA's shares of <S_k, g> and |S_k|^2 for every frame, slices in order
+    for (int k0 = 0; k0 < F; k0 += CHUNK) {
+        if (!one_chunk) load_chunk(k0);              // (a second round trip per chunk for clips of several chunks)
 #pragma unroll
-    for (int jj = 0; jj < FB; ++jj) {                // this CTA's shares of <S_k, g> and |S_k|^2, slices in order
-        float d = 0.f, qq = 0.f;
+        for (int jj = 0; jj < FB; ++jj) {
+            float d = 0.f, qq = 0.f;
 #pragma unroll
-        for (int sl = 0; sl < SL; ++sl) {
-            const float4 x = v[sl][jj], g = gl[sl];
-            d = fmaf(x.x, g.x, d); d = fmaf(x.y, g.y, d); d = fmaf(x.z, g.z, d); d = fmaf(x.w, g.w, d);
-            qq = fmaf(x.x, x.x, qq); qq = fmaf(x.y, x.y, qq); qq = fmaf(x.z, x.z, qq); qq = fmaf(x.w, x.w, qq);
+            for (int sl = 0; sl < SL; ++sl) {
+                const float4 x = v[sl][jj], g = gl[sl];
+                d = fmaf(x.x, g.x, d); d = fmaf(x.y, g.y, d); d = fmaf(x.z, g.z, d); d = fmaf(x.w, g.w, d);
+                qq = fmaf(x.x, x.x, qq); qq = fmaf(x.y, x.y, qq); qq = fmaf(x.z, x.z, qq); qq = fmaf(x.w, x.w, qq);
+            }
+            d = warp_sum(d);
+            qq = warp_sum(qq);
+            const int kk = k0 + w + jj * kNormWarps;
+            if (lane == 0 && kk < F) { s_D[kk] = d; s_Q[kk] = qq; }
         }
-        d = warp_sum(d);
-        qq = warp_sum(qq);
-        const int kk = w + jj * kNormWarps;
-        if (lane == 0) { s_D[kk] = d; s_Q[kk] = qq; }
     }
     if (w == 0) {
         float gg = 0.f;
@@ -394,7 +412,7 @@ k_frame_stats_cluster(const float* S, int F, int C, int nsl, int* hdr, int* out_
         // Eq. (auto_anchor): a* = arg max_k <S_k, g> / (|S_k| |g|), lowest frame on ties; ranks added in rank order
         float best = -INFINITY;
         int idx = 0x7fffffff;
-        if (tid < F) {
+        if (tid < F) {                               // F <= kStatClusterMaxF = the CTA's 256 threads
             float D = s_D[tid], Q = s_Q[tid], G = s_G;
             for (int r = 0; r < kStatCluster - 1; ++r) { D += s_x[r][tid]; Q += s_x[r][F + tid]; G += s_x[r][2 * F]; }
             best = D * (1.0f / fmaxf(sqrtf(G), kNormFloor)) * (1.0f / fmaxf(sqrtf(Q), kNormFloor));
@@ -453,11 +471,11 @@ cudaError_t launch_norm_sum(const Problem& p, const Scratch& s, cudaStream_t st)
 
 cudaError_t launch_frame_stats(const Problem& p, const Scratch& s, int* out_anchor, cudaStream_t st) {
     if (p.anchor_mode != 0) return cudaSuccess;                // fixed anchors need no statistics
-    if (p.C % 4 == 0 && p.nsl <= 4 * kStatCluster) {           // small enough for the single-cluster kernel?
+    if (p.C % 4 == 0 && p.nsl <= 4 * kStatCluster && p.F <= kStatClusterMaxF) {   // the single-cluster kernel takes it
         const int sl = (p.nsl + kStatCluster - 1) / kStatCluster;          // slices per CTA: 1 .. 4
-        if (sl <= 1 && p.F <= kNormWarps * 16) return launch_stats_cluster_t<1>(p, s, out_anchor, st);
-        if (sl <= 2 && p.F <= kNormWarps * 8) return launch_stats_cluster_t<2>(p, s, out_anchor, st);
-        if (sl <= 4 && p.F <= kNormWarps * 4) return launch_stats_cluster_t<4>(p, s, out_anchor, st);
+        if (sl <= 1) return launch_stats_cluster_t<1>(p, s, out_anchor, st);
+        if (sl <= 2) return launch_stats_cluster_t<2>(p, s, out_anchor, st);
+        return launch_stats_cluster_t<4>(p, s, out_anchor, st);
     }
     if (p.C % 4 == 0)
         return launch_pdl(k_frame_stats<4>, dim3(p.nsl), dim3(kNormThreads), st, (const float*)s.S, p.F, p.C, p.nsl,
