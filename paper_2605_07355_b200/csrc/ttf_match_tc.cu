@@ -155,7 +155,7 @@ __global__ void __launch_bounds__(kTcThreads)
 k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
            int F, int H, int W, int C, float t, AnchorSrc asrc, int pieces,
            float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt,
-           int wait_limit)
+           int wait_limit, int tx_extra)
 {
     using S = TcShape<R>;
     extern __shared__ unsigned char dyn_raw[];
@@ -232,7 +232,7 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
                 if (*(volatile int*)&s_err) break;
                 unsigned char* sa = dyn + (size_t)s * S::STAGE;
                 const int c0 = (st0 + it) * kTcKC;
-                mbar_arrive_expect_tx(&bar_full[s], kTcABytes + S::BBOX);
+                mbar_arrive_expect_tx(&bar_full[s], kTcABytes + S::BBOX + (uint32_t)tx_extra);   // (extra: test hook only)
                 tma_load_4d(sa, &mapA, c0, x0, y, k0, &bar_full[s]);
                 tma_load_4d(sa + kTcABytes, &mapB, c0, x0 - R, y - R, a, &bar_full[s]);
                 issued = it + 1;
@@ -487,7 +487,7 @@ static cudaError_t launch_tc_t(const Problem& p, const Scratch& s, int* out_anch
     }
     cfg.attrs = attr; cfg.numAttrs = n;
     return cudaLaunchKernelEx(&cfg, k_match_tc<R>, mapA, mapB, p.F, p.H, p.W, p.C, p.t, make_anchor_src(p, s, out_anchor),
-                              pieces, shat, dst, keep, s.cnt, wait_poll_limit());
+                              pieces, shat, dst, keep, s.cnt, wait_poll_limit(), wait_tx_extra());
 }
 
 cudaError_t launch_match_tc(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,

@@ -44,6 +44,37 @@ def test_copy_wait_runs_out_then_the_next_call_is_clean():
         check_clip(X, 1, 0.7, stream=st)                                 # and it still equals the oracle
 
 
+@pytest.mark.parametrize("C", [256, 2048])
+def test_tensor_core_pipeline_gives_up_and_recovers(C):
+    """the tcgen05 matching kernel under the same hook: its copy barriers never complete, so its MMA issuer, its
+    epilogue warps and then its producer run out of polls; the CTAs (alone for C = 256, in clusters of 8 for
+    C = 2048) still meet at their barriers, free their tensor memory and return; the query reports the time-out
+    and the next call is clean"""
+    X = corr_clip(6, 6, 7, C, seed=79, dtype="bf16")
+    Xd = to_device(X)
+    st = torch.cuda.Stream()
+    P.ttf_set_match_kernel(2)
+    try:
+        ref = P.ttf_query(Xd, 1, 0.7, stream=st)
+        assert P.ttf_last_device_status(st) == B.TTF_OK
+        P.ttf_debug_set_wait(32, 16)
+        try:
+            P.ttf_query(Xd, 1, 0.7, stream=st)
+            assert P.ttf_last_device_status(st) == B.TTF_ERR_TIMEOUT
+            _, cnt, _ = P.ttf_compress(Xd, 1, 0.7, stream=st)
+            assert P.ttf_last_device_status(st) == B.TTF_ERR_TIMEOUT and int(cnt.item()) == -1
+        finally:
+            P.ttf_debug_set_wait()
+        again = P.ttf_query(Xd, 1, 0.7, stream=st)
+        assert P.ttf_last_device_status(st) == B.TTF_OK
+        for k in ref:
+            assert torch.equal(ref[k], again[k]), k
+        with torch.cuda.stream(st):
+            check_clip(X, 1, 0.7, stream=st)
+    finally:
+        P.ttf_set_match_kernel(0)
+
+
 def test_status_of_caller_owned_and_built_in_scratch():
     X = corr_clip(4, 5, 5, 128, seed=78, dtype="bf16")
     Xd = to_device(X)
