@@ -95,7 +95,7 @@ class ClockSampler:
     REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
                0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
 
-    def __init__(self, torch_device: int, period_s: float = 0.02):
+    def __init__(self, torch_device: int, period_s: float = 0.004):
         self.samples = []           # (time, sm_mhz, reasons bitmask)
         self.period = period_s
         self.handle = None

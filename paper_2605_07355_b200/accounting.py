@@ -44,7 +44,7 @@ def kernel_bytes(kind: str, F: int, N: int, C: int, itemsize: int, count: int) -
 
 def pipeline_dram_bytes_model(F: int, N: int, C: int, itemsize: int, count: int, lanes: int, fixed_anchor: bool = False) -> int:
     """DRAM bytes one clip moves in the pipeline as scheduled (confirmed with the profiler's DRAM counters over a
-    whole step: 93.6 / 160.2 / 178.3 MB per 8B-shaped clip for 1 / 2 / 8 clips in flight, 113.7 MB with a fixed
+    whole step: 93.8 / 153.4 / 172.7 MB per 8B-shaped clip for 1 / 2 / 8 clips in flight, 113.7 MB with a fixed
     anchor).  With one clip in flight the matching pass and the gather find the clip in L2, so it is read once; with
     two or more in flight the clips displace one another, and the second pass over X (which only the automatic anchor
     of Eq. auto_anchor needs) and the gather's rows come from DRAM again.  Output rows, positions and the small
