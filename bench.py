@@ -54,6 +54,9 @@ def parse_args():
                     help="profiling aid: after the warm-up run ONE step between cudaProfilerStart/Stop and exit without "
                          "timing anything (for `ncu --replay-mode range`, which measures the overlapped kernels of the "
                          "step as one workload)")
+    ap.add_argument("--extensions", action="store_true",
+                    help="time the extension entry points (restore, streaming segment, histogram, mean fuse) instead of "
+                         "the compression pass and print one JSON line with their roofline fractions")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=5)
@@ -219,6 +222,88 @@ def reference_arm(args):
     print(json.dumps(line), flush=True)
 
 
+def extensions_arm(args):
+    """Times the extension entry points one by one on args.workload: every call on a clip that is cold in L2 (the
+    calls rotate over args.clips distinct clips, together larger than L2), CUDA events on the launching stream.
+    Bytes are the algorithmic ones of each operation; the fraction is against the measured copy rate."""
+    import torch
+    from paper_2605_07355_b200 import build as B
+    from paper_2605_07355_b200 import clips
+    import paper_2605_07355_b200 as P
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    B.build()
+    P.lib()
+    spec = clips.CONFIGS[args.workload]
+    t = spec.t if args.threshold is None else args.threshold
+    F, H, W, C, N = spec.F, spec.H, spec.W, spec.C, spec.H * spec.W
+    row = C * spec.itemsize
+    st = torch.cuda.Stream(device=dev)
+    X, Q, comp, Ls = [], [], [], []
+    for j in range(args.clips):
+        Xn = clips.make_clip(spec, spec.seed + j)
+        th = torch.from_numpy(Xn if spec.dtype == "f32" else Xn.view(np.int16))
+        X.append((th if spec.dtype == "f32" else th.view(torch.bfloat16)).to(dev))
+    with torch.cuda.stream(st):
+        for x in X:
+            Q.append(P.ttf_query(x, spec.r, t, stream=st))
+            toks, cnt, _ = P.ttf_compress(x, spec.r, t, stream=st)
+            L = int(cnt.item())
+            Ls.append(L)
+            comp.append(toks[:L].clone())
+    torch.cuda.synchronize()
+    Lm = float(np.mean(Ls))
+    fused = F * N - Lm
+
+    def timed(call):
+        # warm pass (allocations, attribute set-up), then the pass over all clips captured in a CUDA graph, so that
+        # the host cost of the Python calls stays outside the timed region
+        with torch.cuda.stream(st):
+            for j in range(len(X)):
+                call(j)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            for j in range(len(X)):
+                call(j)
+        reps = max(3, args.steps // 10)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(st):
+            g.replay()
+            e0.record(st)
+            for _ in range(reps):
+                g.replay()
+            e1.record(st)
+        torch.cuda.synchronize()
+        del g
+        return e0.elapsed_time(e1) * 1e3 / (reps * len(X))
+
+    pk_gbs, pk_src = peaks()
+    out = {}
+
+    def entry(name, us, nbytes, note):
+        gbs = nbytes / us * 1e-3
+        out[name] = {"us_per_clip": round(us, 2), "bytes_per_clip": int(nbytes), "achieved_gbs": round(gbs, 1),
+                     "frac_of_copy_rate": round(gbs / pk_gbs, 3), "bytes": note}
+
+    us = timed(lambda j: P.ttf_restore(comp[j], F, H, W, Q[j]["anchor"], Q[j]["keep"], Q[j]["dst"], stream=st))
+    entry("ttf_restore", us, Lm * row + F * N * row + F * N * (1 + 4 + 4),
+          "L' rows read, F*N rows written, keep + dst read, row_index written")
+    us = timed(lambda j: P.ttf_compress_segment(X[j], spec.r, t, 0, stream=st))
+    seg_keep = float(np.mean([int(P.ttf_compress_segment(x, spec.r, t, 0, stream=st)[1].item()) for x in X[:4]]))
+    entry("ttf_compress_segment", us, F * N * row + seg_keep * (row + 12), "X read once, preserved rows and positions written")
+    us = timed(lambda j: P.ttf_sim_histogram(Q[j]["best_sim"], Q[j]["anchor"], F, H, W, 256, stream=st))
+    entry("ttf_sim_histogram", us, F * N * 4 + 256 * 4, "best_sim read, 256 counts written")
+    us = timed(lambda j: P.ttf_compress_mean(X[j], spec.r, t, stream=st))
+    entry("ttf_compress_mean", us, F * N * row + Lm * (row + 12) , "X read once, L' rows and positions written "
+          "(the fused rows' second read for the means is traffic above that)")
+    print(json.dumps({"extensions": out, "workload": workload_config(spec, t, args.clips, 1, F * N * args.clips)["workload"],
+                      "clips": args.clips, "mean_L": Lm, "mean_fused": fused,
+                      "peak_hbm_gbs": pk_gbs, "peak_source": pk_src,
+                      "timing": "CUDA events around graph replays of one call per clip on one stream, clips together larger than L2"}))
+
+
 def combine_ranks(ms_local: float, tokens_local: int, device=None):
     """Whole-job figures of a replica run: the slowest rank's time and the tokens of all ranks.  One clip never
     spans ranks, so this all-reduce of two scalars after the timed region is the only communication there is."""
@@ -245,6 +330,9 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         reference_arm(args)
+        return
+    if args.extensions:
+        extensions_arm(args)
         return
 
     import torch

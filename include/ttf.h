@@ -253,6 +253,22 @@ int ttf_sim_histogram(const float* best_sim, const int* anchor, int F, int H, in
                       unsigned int* out_hist, ttf_stream_t stream);
 
 /*
+ * The counts behind the reduction ratio (Sec. 3, after Eq. Lpre: rho = 1 - (N + P) / (F N)) from ttf_query's
+ * outputs.  out_stats [3] (device, 64-bit): [0] = P, the preserved source tokens (so L' = N + P, Eq. Lpre);
+ * [1] = the fused source tokens, (F-1) N - P; [2] = the source tokens whose best similarity lies within `band` of t
+ * (|best_sim - t| < band, evaluated in double on the stored fp32 values; NaN never counts): the decisions that a
+ * different rounding of the similarity could flip.  The anchor frame is excluded from all three.  band >= 0.
+ * ttf_reduction_ratio below turns P into rho on the host.
+ */
+int ttf_stats(const float* best_sim, const unsigned char* keep, const int* anchor, int F, int H, int W, float t,
+              float band, long long* out_stats, ttf_stream_t stream);
+
+/* rho = 1 - (N + P) / (F N)  (Sec. 3, after Eq. Lpre).  Host arithmetic; N = H * W. */
+static inline double ttf_reduction_ratio(long long P, int F, int N) {
+    return 1.0 - ((double)N + (double)P) / ((double)F * (double)N);
+}
+
+/*
  * The same pass for callers whose tensors live in HOST memory (all four pointers are host pointers; pinned
  * memory makes the copies asynchronous).  Copies features to the device, runs ttf_compress, copies L' and the
  * first L' rows of tokens and positions back, and returns after synchronising.  Device staging buffers are

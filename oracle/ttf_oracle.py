@@ -166,6 +166,28 @@ def sim_histogram(s_hat_f32: np.ndarray, F: int, N: int, a: int, bins: int) -> n
     return hist
 
 
+def stats(s_hat_f32: np.ndarray, keep: np.ndarray, F: int, N: int, a: int, t: float, band: float):
+    """Sec. 3, after Eq. Lpre: rho = 1 - (N + P) / (F N).  Returns (P, fused, in_band, rho) over the source tokens:
+    P preserved, fused = (F-1) N - P, in_band = |s_hat - t| < band on the stored fp32 similarities and the fp32
+    threshold, compared in double.  Plain loops, one token at a time."""
+    s = np.asarray(s_hat_f32, dtype=np.float32).reshape(F, N)
+    kp = np.asarray(keep).reshape(F, N)
+    tt = float(np.float32(t))
+    bb = float(np.float32(band))
+    P = fused = in_band = 0
+    for k in range(F):
+        if k == a:
+            continue
+        for i in range(N):
+            if kp[k, i]:
+                P += 1
+            else:
+                fused += 1
+            if abs(float(s[k, i]) - tt) < bb:
+                in_band += 1
+    return P, fused, in_band, 1.0 - (N + P) / (F * N)
+
+
 def compress_segment(X: np.ndarray, r: int, t: float, frame_base: int, forced_keep: Optional[np.ndarray] = None):
     """Discussion D3 (rolling anchor): frame 0 is the anchor of the segment and is not emitted; returns
     (tokens[P, C], pos[P, 3] with the frame coordinate frame_base + k - 1, P)."""

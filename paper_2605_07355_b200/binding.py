@@ -22,7 +22,7 @@ EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
     "ttf_query_static", "ttf_compress_ex", "ttf_query_ex", "ttf_compress_segment", "ttf_restore",
-    "ttf_sim_histogram", "ttf_compress_batch", "ttf_compress_batch_ex", "ttf_profile_stages", "ttf_compress_mean", "ttf_compress_host_batch",
+    "ttf_sim_histogram", "ttf_stats", "ttf_compress_batch", "ttf_compress_batch_ex", "ttf_profile_stages", "ttf_compress_mean", "ttf_compress_host_batch",
     "ttf_set_schedule", "ttf_set_match_kernel", "ttf_last_device_status", "ttf_workspace_status", "ttf_debug_set_wait", "ttf_debug_func_attr_needed",
 ]
 TTF_ERR_TIMEOUT, TTF_ERR_STATIC_LIMIT = 5, 6
@@ -110,6 +110,8 @@ def lib() -> ctypes.CDLL:
         L.ttf_compress_segment.argtypes = [vp] + shape + [f, i, i, vp, vp, vp, vp]
         L.ttf_restore.restype = i
         L.ttf_restore.argtypes = [vp, sz, i, i, i, vp, vp, vp, vp, vp, vp]
+        L.ttf_stats.restype = i
+        L.ttf_stats.argtypes = [vp, vp, vp, i, i, i, ctypes.c_float, ctypes.c_float, vp, vp]
         L.ttf_sim_histogram.restype = i
         L.ttf_sim_histogram.argtypes = [vp, vp, i, i, i, i, vp, vp]
         L.ttf_query_static.restype = i
@@ -401,6 +403,23 @@ def ttf_sim_histogram(best_sim: torch.Tensor, anchor: torch.Tensor, F: int, H: i
     if rc != TTF_OK:
         raise TTFError(rc, "ttf_sim_histogram")
     return hist
+
+
+def ttf_stats(best_sim: torch.Tensor, keep: torch.Tensor, anchor: torch.Tensor, F: int, H: int, W: int, t: float,
+              band: float = 1e-4, stream=None) -> torch.Tensor:
+    """ttf_stats: int64 [3] on the device = (P preserved, fused, in-band source tokens).  Does not synchronise."""
+    dev = best_sim.device
+    out = torch.empty(3, dtype=torch.int64, device=dev)
+    with torch.cuda.device(dev):
+        rc = lib().ttf_stats(_p(best_sim), _p(keep), _p(anchor), F, H, W, float(t), float(band), _p(out), _stream_ptr(stream))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_stats")
+    return out
+
+
+def ttf_reduction_ratio(P_count: int, F: int, N: int) -> float:
+    """rho = 1 - (N + P) / (F N)  (Sec. 3, after Eq. Lpre); the header's inline helper, restated for Python callers."""
+    return 1.0 - (N + P_count) / (F * N)
 
 
 def ttf_compress_host(features: torch.Tensor, r: int, t: float, out_tokens: Optional[torch.Tensor] = None,

@@ -710,6 +710,15 @@ int ttf_sim_histogram(const float* best_sim, const int* anchor, int F, int H, in
     return e == cudaSuccess ? TTF_OK : cuda_fail(e);
 }
 
+int ttf_stats(const float* best_sim, const unsigned char* keep, const int* anchor, int F, int H, int W, float t,
+              float band, long long* out_stats, ttf_stream_t stream) {
+    if (!best_sim || !keep || !anchor || !out_stats || F < 1 || H < 1 || W < 1 || !(band >= 0.0f) || !(t == t))
+        return TTF_ERR_INVALID_ARG;
+    if ((long long)F * H * W >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
+    cudaError_t e = launch_stats(best_sim, keep, anchor, F, H * W, t, band, out_stats, (cudaStream_t)stream);
+    return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+}
+
 int ttf_query_static(const void* features, int F, int H, int W, int C, int r, float t, int dtype,
                      int* out_anchor, unsigned char* out_keep, int* out_dst, float* out_best_sim,
                      int* out_fuse_cnt, ttf_stream_t stream) {

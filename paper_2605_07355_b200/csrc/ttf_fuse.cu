@@ -12,6 +12,8 @@ namespace ttf {
 
 constexpr int kFuseThreads = 256;
 constexpr int kFuseWarps = kFuseThreads / 32;
+constexpr int kFuseCand = 2;                 // candidates a thread tests per round (512 per CTA: one round for F <= 57 at r = 1)
+constexpr int kRows = 8;                     // rows a thread has in flight
 
 // fp32 -> storage type, round to nearest even
 template <typename T> struct Narrow;
@@ -51,26 +53,31 @@ template <> struct Storer<bf16_t, 1> {
     static __device__ __forceinline__ void store(bf16_t* p, const float (&x)[1]) { p[0] = Narrow<bf16_t>::from(x[0]); }
 };
 
-// CTA = (anchor cell j, slice of kFuseThreads * V channels).  Candidates are taken kFuseThreads at a time in
-// ascending flat order; the ones fused into j are packed, in that order, into a list in shared memory (ballot +
-// prefix over the warps), then every thread adds the listed rows to its V channels.
+// CTA = (anchor cell j, slice of kFuseThreads * V channels): small CTAs, so that all of them are resident at once
+// (a 32-frame 16 x 16 clip of 4096 bf16 channels makes 2048 of them, 14 per SM) and the time of the kernel is the
+// time of one CTA rather than a sum over waves.  Candidates are taken kFuseCand per thread and round in ascending
+// flat order; the ones fused into j are packed, in that order, into a list in shared memory (prefix sum over the
+// CTA), then every thread adds the listed rows to its V channels, kRows loads in flight.
 template <typename T, int V>
 __global__ void __launch_bounds__(kFuseThreads)
 k_fuse_mean(const T* __restrict__ X, int F, int H, int W, int C, int r, const int* __restrict__ hdr,
             const unsigned char* __restrict__ keep, const int* __restrict__ dst, T* __restrict__ out_tokens, int nslices)
 {
     using L = Loader<T, V>;
-    __shared__ int s_list[kFuseThreads];
-    __shared__ int s_warp[kFuseWarps];
+    constexpr int kRound = kFuseCand * kFuseThreads;
+    __shared__ int s_list[kRound];
+    __shared__ int s_cnt[kFuseCand][kFuseWarps];
     const int N = H * W;
     const int j = blockIdx.x / nslices, slice = blockIdx.x - j * nslices;
     const int tid = threadIdx.x, lane = tid & 31, w = tid >> 5;
-    const int a = hdr[HDR_ANCHOR];
+    pdl_launch_dependents();
+    pdl_wait();                                  // the gather has written the anchor rows this kernel overwrites
+    const int a = __ldcg(hdr + HDR_ANCHOR);
     const int y = j / W, x = j - y * W;
     const int y_lo = max(0, y - r), y_hi = min(H - 1, y + r);
     const int x_lo = max(0, x - r), x_hi = min(W - 1, x + r);
     const int nx = x_hi - x_lo + 1, wsz = (y_hi - y_lo + 1) * nx;       // window ∩ grid, ascending cell index
-    const long long ncand = (long long)(F - 1) * wsz;
+    const int ncand = (F - 1) * wsz;                                    // < 2^31: checked by the host
     const int c0 = (slice * kFuseThreads + tid) * V;
     const bool on = c0 < C;
 
@@ -81,43 +88,55 @@ k_fuse_mean(const T* __restrict__ X, int F, int H, int W, int C, int r, const in
         for (int v = 0; v < V; ++v) acc[v] = 0.f;
     }
     int members = 1;
-    for (long long q0 = 0; q0 < ncand; q0 += kFuseThreads) {
-        const long long q = q0 + tid;
-        int f = -1;
-        if (q < ncand) {
-            const int kk = (int)(q / wsz), e = (int)(q - (long long)kk * wsz);
-            const int k = kk < a ? kk : kk + 1;                          // source frames only
-            const int cell = (y_lo + e / nx) * W + x_lo + e % nx;
-            const int cand = k * N + cell;
-            if (!keep[cand] && dst[cand] == j) f = cand;
-        }
-        const unsigned m = __ballot_sync(0xffffffffu, f >= 0);
-        if (lane == 0) s_warp[w] = __popc(m);
-        __syncthreads();
-        int before = 0, total = 0;
+    for (int q0 = 0; q0 < ncand; q0 += kRound) {
+        int f[kFuseCand], kp[kFuseCand], d[kFuseCand];
+        // all loads first and unconditional (a candidate index beyond the end is clamped to the last one and ignored
+        // below), so that they are in flight together; neighbouring lanes test neighbouring candidates, so that one
+        // load instruction touches few sectors
 #pragma unroll
-        for (int ww = 0; ww < kFuseWarps; ++ww) { const int c = s_warp[ww]; if (ww < w) before += c; total += c; }
-        if (f >= 0) s_list[before + __popc(m & ((1u << lane) - 1u))] = f;
+        for (int h = 0; h < kFuseCand; ++h) {                            // thread t tests q0 + h kFuseThreads + t
+            const int q = min(q0 + h * kFuseThreads + tid, ncand - 1);
+            const int kk = (int)((unsigned)q / (unsigned)wsz), e = q - kk * wsz;
+            const int k = kk < a ? kk : kk + 1;                          // source frames only
+            const int ey = (int)((unsigned)e / (unsigned)nx);
+            f[h] = k * N + (y_lo + ey) * W + x_lo + (e - ey * nx);
+            kp[h] = __ldcg(keep + f[h]);
+            d[h] = __ldcg(dst + f[h]);
+        }
+        unsigned m[kFuseCand];
+#pragma unroll
+        for (int h = 0; h < kFuseCand; ++h) {
+            const bool hit = q0 + h * kFuseThreads + tid < ncand && !kp[h] && d[h] == j;
+            m[h] = __ballot_sync(0xffffffffu, hit);
+            if (!hit) f[h] = -1;
+            if (lane == 0) s_cnt[h][w] = __popc(m[h]);
+        }
+        __syncthreads();
+        int total = 0;                                                   // list position: ascending q = (h, warp, lane)
+        const unsigned lt = (1u << lane) - 1u;
+#pragma unroll
+        for (int h = 0; h < kFuseCand; ++h) {
+#pragma unroll
+            for (int ww = 0; ww < kFuseWarps; ++ww) {
+                if (ww == w && f[h] >= 0) s_list[total + __popc(m[h] & lt)] = f[h];
+                total += s_cnt[h][ww];
+            }
+        }
         __syncthreads();
         if (on) {
-            int e = 0;
-            for (; e + 4 <= total; e += 4) {                             // four rows in flight, added in list order
-                typename L::Raw raw[4];
+            for (int e = 0; e < total; e += kRows) {                     // kRows rows in flight, added in list order
+                typename L::Raw raw[kRows];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) raw[u] = L::load_raw(X + (size_t)s_list[e + u] * C + c0);
+                for (int u = 0; u < kRows; ++u)                          // (beyond the end: the last row again, not added)
+                    raw[u] = L::load_raw(X + (size_t)s_list[min(e + u, total - 1)] * C + c0);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < kRows; ++u) {
                     float v[V];
                     L::unpack(raw[u], v);
+                    const bool in = e + u < total;
 #pragma unroll
-                    for (int c = 0; c < V; ++c) acc[c] += v[c];
+                    for (int c2 = 0; c2 < V; ++c2) acc[c2] = in ? acc[c2] + v[c2] : acc[c2];
                 }
-            }
-            for (; e < total; ++e) {
-                float v[V];
-                L::load(X + (size_t)s_list[e] * C + c0, v);
-#pragma unroll
-                for (int c = 0; c < V; ++c) acc[c] += v[c];
             }
         }
         members += total;
@@ -126,7 +145,7 @@ k_fuse_mean(const T* __restrict__ X, int F, int H, int W, int C, int r, const in
     if (on) {
         const float denom = (float)members;
 #pragma unroll
-        for (int c = 0; c < V; ++c) acc[c] = acc[c] / denom;
+        for (int c2 = 0; c2 < V; ++c2) acc[c2] = acc[c2] / denom;
         Storer<T, V>::store(out_tokens + (size_t)j * C + c0, acc);
     }
 }
@@ -136,11 +155,11 @@ static cudaError_t launch_fuse_mean_t(const Problem& p, const Scratch& s, void* 
     const int per = kFuseThreads * V;
     const int nslices = (p.C + per - 1) / per;
     const long long blocks = (long long)p.N * nslices;
-    if (blocks >= (1LL << 31)) return cudaErrorInvalidConfiguration;
-    k_fuse_mean<T, V><<<(unsigned)blocks, kFuseThreads, 0, st>>>(
-        reinterpret_cast<const T*>(p.X), p.F, p.H, p.W, p.C, p.r, s.hdr, s.keep, s.dst,
-        reinterpret_cast<T*>(out_tokens), nslices);
-    return cudaGetLastError();
+    if (blocks >= (1LL << 31) || (long long)p.F * (2 * p.r + 1) * (2 * p.r + 1) >= (1LL << 31) - kFuseCand * kFuseThreads)
+        return cudaErrorInvalidConfiguration;
+    return launch_pdl(k_fuse_mean<T, V>, dim3((unsigned)blocks), dim3(kFuseThreads), st,
+                      reinterpret_cast<const T*>(p.X), p.F, p.H, p.W, p.C, p.r, (const int*)s.hdr,
+                      (const unsigned char*)s.keep, (const int*)s.dst, reinterpret_cast<T*>(out_tokens), nslices);
 }
 
 // Overwrites rows [0, N) of out_tokens (the anchor block of the compressed sequence) with the means; reads the

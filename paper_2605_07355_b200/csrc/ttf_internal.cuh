@@ -109,6 +109,8 @@ cudaError_t launch_restore(const void* comp, size_t row_bytes, int F, int N, con
                            cudaStream_t st);
 cudaError_t launch_sim_histogram(const float* sim, const int* anchor, int F, int N, int bins, unsigned int* hist,
                                  cudaStream_t st);
+cudaError_t launch_stats(const float* sim, const unsigned char* keep, const int* anchor, int F, int N, float t, float band,
+                         long long* out, cudaStream_t st);
 
 // Optional mean fusion (ttf_fuse.cu; not the paper's method): overwrites the anchor block of out_tokens.
 cudaError_t launch_fuse_mean(const Problem& p, const Scratch& s, void* out_tokens, cudaStream_t st);

@@ -99,6 +99,10 @@ def test_batch_and_variant_entry_points_validate_before_any_cuda_call(lib):
     ms = (ctypes.c_double * 5)()
     assert lib.ttf_profile_stages(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, 0, ms, 5, None) == 1   # reps < 1
     assert lib.ttf_profile_stages(arr, 2, 4, 4, 4, 8, 1, 0.7, 0, arr, arr, arr, 1, None, 5, None) == 1
+    assert lib.ttf_stats(None, fake, fake, 4, 4, 4, 0.7, 1e-4, fake, None) == 1
+    assert lib.ttf_stats(fake, fake, fake, 4, 4, 4, 0.7, -1.0, fake, None) == 1                  # negative band
+    assert lib.ttf_stats(fake, fake, fake, 4, 4, 4, float("nan"), 1e-4, fake, None) == 1
+    assert lib.ttf_stats(fake, fake, fake, 0, 4, 4, 0.7, 1e-4, fake, None) == 1
     assert lib.ttf_set_schedule(9) == 1 and lib.ttf_set_schedule(-1) == 1
     assert lib.ttf_set_schedule(0) == 0
 

@@ -79,3 +79,22 @@ def test_segment_matches_oracle(shape, dtype):
     assert Pn == ref_P == int(keep.sum()) - N
     assert (pos[:Pn].cpu().numpy() == ref_p).all() and (to_bits(toks[:Pn]) == ref_t).all()
     assert Pn == 0 or int(pos[:Pn, 0].min().item()) >= 17
+
+
+@pytest.mark.parametrize("name,band", [("tiny_cal", 1e-2), ("vl2b_cal", 1e-3)])
+def test_stats_match_oracle(name, band):
+    """ttf_stats on the GPU's own query outputs equals the oracle's counts exactly (integers), rho follows."""
+    s = clips.CONFIGS[name]
+    X = clips.make_clip(s)
+    F, H, W = s.F, s.H, s.W
+    N = H * W
+    q = P.ttf_query(to_device(X), s.r, s.t)
+    st = P.ttf_stats(q["best_sim"], q["keep"], q["anchor"], F, H, W, s.t, band)
+    torch.cuda.synchronize()
+    a = int(q["anchor"].item())
+    Pn, fused, in_band, rho = O.stats(q["best_sim"].cpu().numpy(), q["keep"].cpu().numpy(), F, N, a, s.t, band)
+    assert st.tolist() == [Pn, fused, in_band]
+    assert in_band > 0 and Pn + fused == (F - 1) * N
+    assert P.ttf_reduction_ratio(int(st[0]), F, N) == rho
+    toks, cnt, pos = P.ttf_compress(to_device(X), s.r, s.t)
+    assert int(cnt.item()) == N + Pn                                  # L' = N + P (Eq. Lpre)

@@ -415,3 +415,29 @@ def test_bf16_rounding_helper_is_round_to_nearest_even():
     assert (O.round_to_bf16_bits(x.astype(np.float64)) == rne).all()
     ties = np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -1.0 - 3 * 2.0 ** -8])
     assert O.round_to_bf16_bits(ties).tolist() == [0x3F80, 0x3F82, 0xBF82]
+
+
+def test_stats_reduction_ratio_closed_forms_and_count_identity():
+    """Sec. 3 (after Eq. Lpre): rho = 1 - (N + P) / (F N).  Identical frames fuse every source token: P = 0 and
+    rho = 1 - 1/F exactly; a threshold nothing exceeds keeps everything: rho = 0; on a generic clip N + P equals the
+    length of the compressed sequence the compaction step returns, and the band count equals a vectorised count."""
+    rng = np.random.default_rng(5)
+    F, H, W, C = 6, 3, 4, 16
+    N = H * W
+    frame = rng.standard_normal((H, W, C)).astype(np.float32)
+    X = np.broadcast_to(frame, (F, H, W, C)).copy()
+    R = O.compress(X, 1, 0.7)
+    P, fused, band, rho = O.stats(R.s_hat.astype(np.float32), R.keep, F, N, R.anchor, 0.7, 1e-4)
+    assert (P, fused) == (0, (F - 1) * N) and rho == 1.0 - 1.0 / F
+    R = O.compress(X, 1, 2.0)
+    P, fused, band, rho = O.stats(R.s_hat.astype(np.float32), R.keep, F, N, R.anchor, 2.0, 1e-4)
+    assert (P, fused, band) == ((F - 1) * N, 0, 0) and rho == 0.0
+    X = rng.standard_normal((F, H, W, C)).astype(np.float32) * 0.6 + frame
+    R = O.compress(X, 1, 0.6)
+    s32 = R.s_hat.astype(np.float32)
+    P, fused, band, rho = O.stats(s32, R.keep, F, N, R.anchor, 0.6, 0.05)
+    assert N + P == R.count and P + fused == (F - 1) * N and 0 < P < (F - 1) * N
+    src = np.arange(F) != R.anchor
+    want = int((np.abs(s32.reshape(F, N)[src].astype(np.float64) - float(np.float32(0.6))) < float(np.float32(0.05))).sum())
+    assert band == want and band > 0
+    assert abs(rho - (1.0 - R.count / (F * N))) < 1e-15
