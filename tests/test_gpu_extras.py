@@ -38,6 +38,28 @@ def test_restore_matches_oracle(shape, dtype):
     assert (full2.cpu().numpy() == payload.cpu().numpy()[ref_idx]).all()
 
 
+@pytest.mark.parametrize("offset", [0, 1, 3, 13])
+def test_restore_flag_counts_from_any_alignment(offset):
+    """The index step counts the flags of earlier frames 16 per load between an unaligned head and tail: odd N,
+    many frames, the flag array at every kind of offset from a 16-byte boundary, non-0/1 flag values."""
+    F, H, W, C = 45, 5, 7, 16
+    N = H * W
+    X = corr_clip(F, H, W, C, seed=123, dtype="f32")
+    q = P.ttf_query(to_device(X), 1, 0.6)
+    toks, cnt, _ = P.ttf_compress(to_device(X), 1, 0.6)
+    torch.cuda.synchronize()
+    L = int(cnt.item())
+    buf = torch.zeros(F * N + 32, dtype=torch.uint8, device="cuda")
+    keep_view = buf[offset:offset + F * N]
+    keep_view.copy_(q["keep"].view(-1) * 255)                        # any non-zero value is a set flag
+    full, idx = P.ttf_restore(toks[:L].contiguous(), F, H, W, q["anchor"], keep_view, q["dst"])
+    torch.cuda.synchronize()
+    keep, dst, a = q["keep"].cpu().numpy(), q["dst"].cpu().numpy(), int(q["anchor"].item())
+    ref_full, ref_idx = O.restore(to_bits(toks[:L]), keep, dst, F, N, a)
+    assert (idx.cpu().numpy() == ref_idx).all()
+    assert (to_bits(full) == ref_full).all()
+
+
 @pytest.mark.parametrize("bins", [1, 16, 100])
 def test_histogram_matches_oracle(bins):
     s = clips.CONFIGS["vl2b_cal"]
