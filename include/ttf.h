@@ -52,7 +52,8 @@ typedef enum {
     TTF_ERR_WORKSPACE = 3,     /* caller workspace NULL, smaller than ttf_workspace_bytes or not 256-aligned */
     TTF_ERR_CUDA = 4,          /* a CUDA runtime call failed (see ttf_last_cuda_error)                       */
     TTF_ERR_TIMEOUT = 5,       /* device status only: a kernel gave up on one of its bounded waits           */
-    TTF_ERR_STATIC_LIMIT = 6   /* ttf_query_static: the clip needs more scratch than TTF_STATIC_SCRATCH_BYTES */
+    TTF_ERR_STATIC_LIMIT = 6,  /* ttf_query_static: the clip needs more scratch than TTF_STATIC_SCRATCH_BYTES */
+    TTF_ERR_BOUNDS = 7         /* device status only, checked build: a kernel computed an index outside its array */
 } ttf_status;
 
 /* anchor rule: Eq. (auto_anchor), or the fixed first / last frame anchors compared in Table 1 and ablation A2,
@@ -86,7 +87,8 @@ int ttf_last_cuda_error(void);
  * waits inside the kernels are waits of a warp for its own asynchronous copies; each is bounded, and a warp whose
  * wait runs out stops copying and sets an error word in the call's scratch, which the first kernel of every call
  * clears.  ttf_last_device_status synchronises `stream`, reads the error word(s) of the last call enqueued on it (for
- * a batch call: of every clip of the batch) and stores TTF_OK or TTF_ERR_TIMEOUT in *host_status.  ttf_compress also
+ * a batch call: of every clip of the batch) and stores TTF_OK or TTF_ERR_TIMEOUT (in the checked build also
+ * TTF_ERR_BOUNDS) in *host_status.  ttf_compress also
  * reports the condition as out_count = -1; the query entry points have no other channel than this one.  The return
  * value is the status of the status query itself.  ttf_workspace_status is the same for calls that ran on
  * caller-owned scratch (`workspace` as passed to the _ws entry point; NULL = the built-in array of ttf_query_static).
@@ -102,9 +104,16 @@ int ttf_workspace_status(const void* workspace, ttf_stream_t stream, int* host_s
  * can be exercised without a fault or a hang.  Process-wide.
  * ttf_debug_func_attr_needed: the per-(function, device) table behind the kernels' dynamic shared memory limits;
  * returns 1 when (key, device) had not been recorded with at least `bytes` before, and records it.
+ * ttf_debug_set_check_slack: only in the checked build of the library (the same sources compiled with -DTTF_DEBUG:
+ * every global store whose index a kernel computes is preceded by a range test; an index outside its array is
+ * recorded, the store is skipped, nothing traps, and the device status becomes TTF_ERR_BOUNDS).  `slack` >= 0 lowers
+ * every limit of those tests by that many elements, so that valid indices at the end of an array are reported and
+ * skipped: the reporting path can be exercised with all accesses still in bounds.  The normal build returns
+ * TTF_ERR_UNSUPPORTED.
  */
 int ttf_debug_set_wait(int poll_limit, int tx_extra_bytes);
 int ttf_debug_func_attr_needed(const void* key, int device, size_t bytes);
+int ttf_debug_set_check_slack(int slack);
 
 /*
  * Scratch bytes one call needs for a clip of this shape (per-token inverse norms, per-frame channel sums,

@@ -23,9 +23,9 @@ EXPORTS = [
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
     "ttf_query_static", "ttf_compress_ex", "ttf_query_ex", "ttf_compress_segment", "ttf_restore",
     "ttf_sim_histogram", "ttf_stats", "ttf_compress_batch", "ttf_compress_batch_ex", "ttf_profile_stages", "ttf_compress_mean", "ttf_compress_host_batch",
-    "ttf_set_schedule", "ttf_set_match_kernel", "ttf_last_device_status", "ttf_workspace_status", "ttf_debug_set_wait", "ttf_debug_func_attr_needed",
+    "ttf_set_schedule", "ttf_set_match_kernel", "ttf_last_device_status", "ttf_workspace_status", "ttf_debug_set_wait", "ttf_debug_func_attr_needed", "ttf_debug_set_check_slack",
 ]
-TTF_ERR_TIMEOUT, TTF_ERR_STATIC_LIMIT = 5, 6
+TTF_ERR_TIMEOUT, TTF_ERR_STATIC_LIMIT, TTF_ERR_BOUNDS = 5, 6, 7
 TTF_ANCHOR_AUTO, TTF_ANCHOR_FIRST, TTF_ANCHOR_LAST, TTF_ANCHOR_EXPLICIT = 0, 1, 2, 3
 TTF_ORDER_ANCHOR_FIRST, TTF_ORDER_NATURAL = 0, 1
 
@@ -82,6 +82,8 @@ def lib() -> ctypes.CDLL:
         L.ttf_last_device_status.argtypes = [vp, ctypes.POINTER(i)]
         L.ttf_workspace_status.restype = i
         L.ttf_workspace_status.argtypes = [vp, vp, ctypes.POINTER(i)]
+        L.ttf_debug_set_check_slack.restype = i
+        L.ttf_debug_set_check_slack.argtypes = [i]
         L.ttf_debug_set_wait.restype = i
         L.ttf_debug_set_wait.argtypes = [i, i]
         L.ttf_debug_func_attr_needed.restype = i
@@ -241,6 +243,11 @@ def ttf_debug_set_wait(poll_limit: int = 1 << 18, tx_extra_bytes: int = 0) -> No
     rc = lib().ttf_debug_set_wait(int(poll_limit), int(tx_extra_bytes))
     if rc != TTF_OK:
         raise TTFError(rc, "ttf_debug_set_wait")
+
+
+def ttf_debug_set_check_slack(slack: int = 0) -> int:
+    """ttf_debug_set_check_slack: returns the status (TTF_ERR_UNSUPPORTED = 2 from the normal build)."""
+    return int(lib().ttf_debug_set_check_slack(int(slack)))
 
 
 def ttf_set_match_kernel(which: int = 0) -> None:

@@ -139,7 +139,7 @@ k_norm_sum(const T* __restrict__ X, int F, int N, int C, int nq,
             float s = 0.f;
 #pragma unroll
             for (int r2 = 0; r2 < RG; ++r2) s += sm[r2][idx];
-            S[(size_t)k * C + c] = s;
+            if (in_bounds(hdr, 1, (long long)k * C + c, (long long)F * C)) S[(size_t)k * C + c] = s;
         }
     }
     if (q == 0 && tid == 0) cnt[k] = 0;             // survivor counters start at zero for the matching kernel

@@ -214,10 +214,21 @@ static int clear_control_blocks(void* ws, size_t stride, int n, cudaStream_t st)
     return e == cudaSuccess ? TTF_OK : cuda_fail(e);
 }
 
+// Checked build: the slack by which every index limit of the next calls is lowered (test hook, normally zero).
+#ifdef TTF_DEBUG
+static std::atomic<int> g_check_slack{0};
+__global__ void k_set_word(int* word, int value) { *word = value; }
+#endif
+
 // steps shared by compress and query: norms + frame sums, anchor, matching + gate
 static int run_front(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,
                      unsigned char* keep, cudaStream_t st) {
     cudaError_t e;
+#ifdef TTF_DEBUG
+    k_set_word<<<1, 1, 0, st>>>(s.hdr + HDR_CHECK_SLACK, g_check_slack.load());
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e);
+#endif
     { ProfScope ps(st, PK_NORM_SUM); e = launch_norm_sum(p, s, st); }
     if (e != cudaSuccess) return cuda_fail(e);
     if (p.anchor_mode == 0) {
@@ -318,6 +329,7 @@ const char* ttf_status_string(int status) {
         case TTF_ERR_CUDA: return "TTF_ERR_CUDA";
         case TTF_ERR_TIMEOUT: return "TTF_ERR_TIMEOUT";
         case TTF_ERR_STATIC_LIMIT: return "TTF_ERR_STATIC_LIMIT";
+        case TTF_ERR_BOUNDS: return "TTF_ERR_BOUNDS";
         default: return "TTF_ERR_UNKNOWN";
     }
 }
@@ -330,7 +342,8 @@ static int read_status_words(const std::vector<const int*>& words, int* host_sta
         int v = 0;
         cudaError_t e = cudaMemcpy(&v, hdr + HDR_ERROR, sizeof(int), cudaMemcpyDeviceToHost);
         if (e != cudaSuccess) return cuda_fail(e);
-        if (v) *host_status = TTF_ERR_TIMEOUT;
+        if (v == 2) *host_status = TTF_ERR_BOUNDS;                   // (checked build only)
+        else if (v && *host_status == TTF_OK) *host_status = TTF_ERR_TIMEOUT;
     }
     return TTF_OK;
 }
@@ -708,6 +721,17 @@ int ttf_sim_histogram(const float* best_sim, const int* anchor, int F, int H, in
     if ((long long)F * H * W >= (1LL << 31)) return TTF_ERR_UNSUPPORTED;
     cudaError_t e = launch_sim_histogram(best_sim, anchor, F, H * W, bins, out_hist, (cudaStream_t)stream);
     return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+}
+
+int ttf_debug_set_check_slack(int slack) {
+#ifdef TTF_DEBUG
+    if (slack < 0) return TTF_ERR_INVALID_ARG;
+    g_check_slack.store(slack);
+    return TTF_OK;
+#else
+    (void)slack;
+    return TTF_ERR_UNSUPPORTED;                  // this build carries no index checks
+#endif
 }
 
 int ttf_stats(const float* best_sim, const unsigned char* keep, const int* anchor, int F, int H, int W, float t,

@@ -126,11 +126,13 @@ k_compact_bulk(const unsigned char* __restrict__ X, size_t row_bytes, int F, int
             if (i < 0) break;                    // cannot happen when cnt matches keep
             f = k * N + i;
         }
-        if (lane < 3) {                          // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
+        // (checked build: the output row and the source row both lie inside their F N rows)
+        const bool row_ok = in_bounds(hdr, 4, j, (long long)F * N) && in_bounds(hdr, 4, f, (long long)F * N);
+        if (lane < 3 && row_ok) {                // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
             const int k = f / N, i = f - k * N, yy = i / W;
             out_pos[(size_t)j * 3 + lane] = pos_base + (lane == 0 ? k + t_off : (lane == 1 ? yy : i - yy * W));
         }
-        if (lane == 0 && !gave_up) {
+        if (lane == 0 && !gave_up && row_ok) {
             for (int pc = 0; pc < pieces; ++pc) {
                 const size_t off = (size_t)pc * kBulkPiece;
                 const uint32_t bytes = (uint32_t)(row_bytes - off < (size_t)kBulkPiece ? row_bytes - off : kBulkPiece);
@@ -214,6 +216,9 @@ k_compact(const unsigned char* __restrict__ X, size_t row_bytes, int F, int H, i
             if (i < 0) break;                              // cannot happen when cnt matches keep
             f = k * N + i;
         }
+        const bool row_ok = in_bounds(const_cast<int*>(hdr), 4, j, (long long)F * N) &&
+                            in_bounds(const_cast<int*>(hdr), 4, f, (long long)F * N);     // (checked build)
+        if (!row_ok) continue;
         if (lane < 3) {                                    // p_{k,i} = (k, y_i, x_i)  (Eq. compress_pos)
             const int k = f / N, i = f - k * N, yy = i / W;
             out_pos[(size_t)j * 3 + lane] = pos_base + (lane == 0 ? k + t_off : (lane == 1 ? yy : i - yy * W));

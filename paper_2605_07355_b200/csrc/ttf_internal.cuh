@@ -17,7 +17,12 @@ constexpr int kStatReplicas = 16;      // copies of the frame statistics, so tha
 // header words of the scratch block
 enum { HDR_ANCHOR = 0,          // anchor frame a*
        HDR_DONE_ALL = 1,        // arrival counter of the statistics CTAs (zero between calls)
-       HDR_ERROR = 2 };         // a bounded wait of this call gave up (cleared by the first kernel of every call)
+       HDR_ERROR = 2,           // 1: a bounded wait of this call gave up; 2: a checked build caught an index outside its
+                                // array (cleared by the first kernel of every call)
+       HDR_CHECK_SLACK = 8,     // checked build: every limit is lowered by this much (test hook; zero otherwise)
+       HDR_CHECK_SITE = 9,      // checked build: kernel site, index (clamped to 31 bits) and limit of the first index
+       HDR_CHECK_INDEX = 10,    // that was out of range
+       HDR_CHECK_LIMIT = 11 };
 
 // Problem description handed to every launcher.
 struct Problem {
@@ -205,6 +210,26 @@ __device__ __forceinline__ void trace_mark_any(int*, int, bool) {}
 __device__ __forceinline__ void trace_mark(int*, int, bool) {}
 __device__ __forceinline__ unsigned long long trace_now() { return 0; }
 __device__ __forceinline__ void trace_acc(int*, int, unsigned long long) {}
+#endif
+
+// Checked build (-DTTF_DEBUG): every global store whose index a kernel computes is guarded by in_bounds().  An
+// index outside [0, limit) raises the status word of the call's scratch to 2, leaves (site, index, limit) of the first
+// offender in the header, and the caller skips the access: nothing traps, the context stays usable, and the host
+// reads TTF_ERR_BOUNDS.  In the normal build the test is the constant true and disappears.
+// Sites: 1 sweep, 2 warp-level / CUDA-core matching, 3 tcgen05 matching, 4 gather rows, 5 gather positions.
+#ifdef TTF_DEBUG
+__device__ __forceinline__ bool in_bounds(int* hdr, int site, long long idx, long long limit) {
+    limit -= __ldcg(hdr + HDR_CHECK_SLACK);
+    if (idx >= 0 && idx < limit) return true;
+    if (atomicCAS(hdr + HDR_ERROR, 0, 2) == 0) {
+        hdr[HDR_CHECK_SITE] = site;
+        hdr[HDR_CHECK_INDEX] = (int)(idx < 0 ? -1 : (idx > 0x7fffffffLL ? 0x7fffffffLL : idx));
+        hdr[HDR_CHECK_LIMIT] = (int)(limit > 0x7fffffffLL ? 0x7fffffffLL : limit);
+    }
+    return false;
+}
+#else
+__device__ __forceinline__ bool in_bounds(int*, int, long long, long long) { return true; }
 #endif
 
 struct bf16_t { uint16_t bits; };   // storage type only: all arithmetic is on the widened fp32 value

@@ -45,7 +45,7 @@ k_match_generic(const T* __restrict__ X, int F, int H, int W, int C, int r, floa
     for (int k = chunk * fchunk + w; k < k_end; k += kMatchWarps) {
         const size_t f = (size_t)k * N + i;
         if (k == a) {                       // anchor tokens are always retained (Eq. mask)
-            if (lane == 0) { shat[f] = 1.0f; dst[f] = i; keep[f] = 1; }
+            if (lane == 0 && in_bounds(asrc.hdr, 2, (long long)f, (long long)FN)) { shat[f] = 1.0f; dst[f] = i; keep[f] = 1; }
             continue;
         }
         const T* xs = X + f * C;
@@ -79,7 +79,7 @@ k_match_generic(const T* __restrict__ X, int F, int H, int W, int C, int r, floa
                 if (s > best || best_j < 0) { best = s; best_j = j; }
             }
         }
-        if (lane == 0) {
+        if (lane == 0 && in_bounds(asrc.hdr, 2, (long long)f, (long long)FN)) {
             const unsigned char kp = !(best > t);
             shat[f] = best; dst[f] = best_j; keep[f] = kp;
             if (kp) atomicAdd(&cnt[k], 1);   // integer count: order-independent
@@ -115,7 +115,7 @@ __device__ __forceinline__ void match_mma_body(const bf16_t* __restrict__ X, int
         trace_mark(asrc.hdr, 4, true);
         return a;
     };
-    match_mma_unit<MT, NT, GRAM, ST>(X, F, H, W, C, r, t, anchor_fn, i, k0, ssq, nslice, shat, dst, keep, cnt, dyn_smem);
+    match_mma_unit<MT, NT, GRAM, ST>(X, F, H, W, C, r, t, anchor_fn, i, k0, ssq, nslice, shat, dst, keep, cnt, asrc.hdr, dyn_smem);
     trace_mark(asrc.hdr, 2, true);
 }
 

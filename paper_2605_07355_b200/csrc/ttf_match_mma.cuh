@@ -120,7 +120,7 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
                                                AnchorFn anchor_fn, int i, int k0, const float* ssq, int nslice,
                                                float* __restrict__ shat, int* __restrict__ dst,
                                                unsigned char* __restrict__ keep, int* __restrict__ cnt,
-                                               unsigned char* dyn_smem)
+                                               int* hdr, unsigned char* dyn_smem)
 {
     constexpr int kMmaStages = ST;
     constexpr int FR = 16 * MT;      // frames per CTA
@@ -268,7 +268,7 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
 
     if (tid < FR) {
         const int k = k0 + tid;
-        if (k < F) {
+        if (k < F && in_bounds(hdr, 2, (long long)k * N + i, (long long)F * N)) {
             const size_t f = (size_t)k * N + i;
             if (k == a) {                           // anchor tokens are always retained (Eq. mask)
                 shat[f] = 1.0f; dst[f] = i; keep[f] = 1;

@@ -368,7 +368,7 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
         epilogue_bar_sync();
         const int kl = m >> 2, dx = m & 3;
         const int k = k0 + kl, x = x0 + dx;
-        if (k < F && x < W) {
+        if (k < F && x < W && in_bounds(asrc.hdr, 3, (long long)k * N + (long long)y * W + x, (long long)F * N)) {
             const size_t f = (size_t)k * N + (size_t)y * W + x;
             if (k == a) {                                  // anchor tokens are always retained (Eq. mask)
                 shat[f] = 1.0f; dst[f] = y * W + x; keep[f] = 1;

@@ -33,6 +33,18 @@ def test_header_symbols_are_exported(lib):
     assert set(names) == set(P.EXPORTS)
 
 
+def test_checked_build_exports_the_same_symbols_and_only_it_takes_the_slack_hook(lib):
+    from paper_2605_07355_b200 import build as B
+    checked = ctypes.CDLL(B.build(checked=True))
+    for n in declared_symbols():
+        assert hasattr(checked, n), n
+    assert lib.ttf_debug_set_check_slack(3) == 2                  # TTF_ERR_UNSUPPORTED: no checks in the normal build
+    assert checked.ttf_debug_set_check_slack(-1) == 1
+    assert checked.ttf_debug_set_check_slack(3) == 0 and checked.ttf_debug_set_check_slack(0) == 0
+    checked.ttf_status_string.restype = ctypes.c_char_p
+    assert checked.ttf_status_string(7) == b"TTF_ERR_BOUNDS"
+
+
 def test_status_strings(lib):
     assert lib.ttf_status_string(0) == b"TTF_OK"
     assert lib.ttf_status_string(1) == b"TTF_ERR_INVALID_ARG"
