@@ -118,7 +118,7 @@ template <int R> struct TcShape {
     static constexpr int BBYTES = NB * 128;
     static constexpr int BBOX = NCAND * 128;              // bytes one B box copy delivers
     static constexpr int STAGE = kTcABytes + BBYTES;
-    static constexpr int STAGES = R == 2 ? 4 : 5;         // two CTAs per SM
+    static constexpr int STAGES = 4;                      // two CTAs per SM with room left for CTAs of other kernels
     static constexpr int TMEM_COLS = NB <= 32 ? 32 : 64;
     static constexpr int WIN = SIDE * SIDE;               // candidates of one source row
 };
@@ -162,7 +162,7 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
     __shared__ uint64_t bar_full[S::STAGES], bar_empty[S::STAGES], bar_acc;
     __shared__ uint32_t s_tmem;
     __shared__ int s_err;
-    __shared__ float s_nb[S::NCAND];                       // squared norms of the candidate rows
+    __shared__ float s_nb[S::NCAND];                       // 1 / norm of the candidate rows
     __shared__ float s_nbp[S::NCAND * 8];                  // ... per 16-byte piece column, before they are added up
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -364,7 +364,7 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
 
     if (warp >= 2 && piece == 0) {
         // ---- epilogue, part 3 (rank 0 of the tile): cosine, arg max over the window clipped to the grid, gate --
-        if (et < S::NCAND) s_nb[et] = nb;
+        if (et < S::NCAND) s_nb[et] = 1.0f / fmaxf(sqrtf(nb), kNormFloor);     // once per candidate row, not once per use
         epilogue_bar_sync();
         const int kl = m >> 2, dx = m & 3;
         const int k = k0 + kl, x = x0 + dx;
@@ -382,8 +382,7 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
                     for (int wx = 0; wx < S::SIDE; ++wx) {     // ascending anchor index among in-grid cells
                         const int yy = y + wy - R, xx = x + wx - R;
                         if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
-                        const float ra = 1.0f / fmaxf(sqrtf(s_nb[wy * S::BW + dx + wx]), kNormFloor);
-                        const float sim = win[wy * S::SIDE + wx] * rs * ra;
+                        const float sim = win[wy * S::SIDE + wx] * rs * s_nb[wy * S::BW + dx + wx];
                         if (sim > best || best_j < 0) { best = sim; best_j = yy * W + xx; }
                     }
                 const unsigned char kp = !(best > t);
