@@ -491,6 +491,8 @@ def main():
     clocks = sampler.summary(w0, w1)
     kernel_ms = P.ttf_profile_stages(devX, spec.r, t, out_tok, out_cnt, out_pos, reps=min(args.steps, 20),
                                      stream=main_stream)
+    # what the plainest read kernel takes on one clip, launched the same way: the floor for a kernel that reads a clip
+    read_floor_us = 1e3 * P.ttf_profile_read_floor(devX, reps=min(args.steps, 20), stream=main_stream)
     torch.cuda.synchronize()
     launches_per_step = 4 * nclips      # sweep (or its stand-in for a fixed anchor), statistics or none, matching, gather
     if amode != 0:
@@ -510,6 +512,9 @@ def main():
                 "frac": achieved / peak_gbs, "peak_source": f"of {peak_kind}",
                 "traffic": traffic, "traffic_note": traffic_note, "csrc_hash": csrc,
                 "algorithmic_bytes_per_launch": kbytes,
+                "read_floor": {"us_per_launch": round(read_floor_us, 3), "gbs": round(clip_bytes / read_floor_us * 1e-3, 1),
+                               "what": "a plain coalesced read kernel over one clip (cold in HBM), launched back to back like "
+                                       "the kernels above: what one launch that reads a clip once can reach"},
                 "kernel_share": {k: kernel_ms[k] / tot for k in kern},
                 "kernel_us": {k: round(kern[k]["us_per_launch"], 3) for k in kern},
                 "kernel_frac": {k: A.kernel_bytes(k, spec.F, spec.N, C, spec.itemsize, int(round(avg_count)))

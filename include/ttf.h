@@ -352,6 +352,17 @@ int ttf_profile_stages(const void* const* features, int nclips, int F, int H, in
                        int dtype, void* const* out_tokens, int* const* out_count, int* const* out_pos_thw,
                        int reps, double* ms_per_launch, int kinds, ttf_stream_t stream);
 
+/*
+ * Measurement aid (no counterpart in the paper): the time of the plainest kernel that reads a buffer once (fully
+ * coalesced 16-byte loads, eight in flight per thread, launched like the kernels of the pass), launched back to back
+ * over `nbuffers` device buffers of `bytes` bytes each (16-byte aligned, a multiple of 16), `reps` rounds after one
+ * warm-up round; *ms_per_launch = time / launches.  With buffers that are together larger than L2 every launch reads
+ * from HBM: this is the floor for any kernel that has to read one clip in one launch, and for clips of some 10 us
+ * of HBM time it lies well below the copy rate of large buffers.  Synchronises `stream`.
+ */
+int ttf_profile_read_floor(const void* const* buffers, int nbuffers, size_t bytes, int reps, double* ms_per_launch,
+                           ttf_stream_t stream);
+
 /* Frees every cached scratch / staging buffer of the calling process (all devices).  Synchronises. */
 int ttf_release(void);
 

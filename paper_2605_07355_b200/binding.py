@@ -22,7 +22,7 @@ EXPORTS = [
     "ttf_status_string", "ttf_last_cuda_error", "ttf_workspace_bytes", "ttf_compress", "ttf_compress_ws",
     "ttf_query", "ttf_query_ws", "ttf_compress_host", "ttf_release", "ttf_profile_begin", "ttf_profile_end",
     "ttf_query_static", "ttf_compress_ex", "ttf_query_ex", "ttf_compress_segment", "ttf_restore",
-    "ttf_sim_histogram", "ttf_stats", "ttf_compress_batch", "ttf_compress_batch_ex", "ttf_profile_stages", "ttf_compress_mean", "ttf_compress_host_batch",
+    "ttf_sim_histogram", "ttf_stats", "ttf_compress_batch", "ttf_compress_batch_ex", "ttf_profile_stages", "ttf_profile_read_floor", "ttf_compress_mean", "ttf_compress_host_batch",
     "ttf_set_schedule", "ttf_set_match_kernel", "ttf_last_device_status", "ttf_workspace_status", "ttf_debug_set_wait", "ttf_debug_func_attr_needed", "ttf_debug_set_check_slack",
 ]
 TTF_ERR_TIMEOUT, TTF_ERR_STATIC_LIMIT, TTF_ERR_BOUNDS = 5, 6, 7
@@ -112,6 +112,8 @@ def lib() -> ctypes.CDLL:
         L.ttf_compress_segment.argtypes = [vp] + shape + [f, i, i, vp, vp, vp, vp]
         L.ttf_restore.restype = i
         L.ttf_restore.argtypes = [vp, sz, i, i, i, vp, vp, vp, vp, vp, vp]
+        L.ttf_profile_read_floor.restype = i
+        L.ttf_profile_read_floor.argtypes = [vp, i, ctypes.c_size_t, i, vp, vp]
         L.ttf_stats.restype = i
         L.ttf_stats.argtypes = [vp, vp, vp, i, i, i, ctypes.c_float, ctypes.c_float, vp, vp]
         L.ttf_sim_histogram.restype = i
@@ -218,6 +220,19 @@ def ttf_profile_stages(features, r: int, t: float, out_tokens, out_count, out_po
     if rc != TTF_OK:
         raise TTFError(rc, "ttf_profile_stages")
     return {k: float(ms[i]) for i, k in enumerate(KERNEL_KINDS[:4])}
+
+
+def ttf_profile_read_floor(buffers, reps: int = 10, stream=None) -> float:
+    """ttf_profile_read_floor: ms per launch of a plain read kernel over each of `buffers` (same size, contiguous)."""
+    nbytes = buffers[0].numel() * buffers[0].element_size()
+    ptrs = (ctypes.c_void_p * len(buffers))(*[b.data_ptr() for b in buffers])
+    ms = ctypes.c_double(0.0)
+    with torch.cuda.device(buffers[0].device):
+        rc = lib().ttf_profile_read_floor(ptrs, len(buffers), ctypes.c_size_t(nbytes), int(reps), ctypes.byref(ms),
+                                          _stream_ptr(stream))
+    if rc != TTF_OK:
+        raise TTFError(rc, "ttf_profile_read_floor")
+    return ms.value
 
 
 def ttf_last_device_status(stream=None) -> int:

@@ -999,6 +999,28 @@ int ttf_profile_stages(const void* const* features, int nclips, int F, int H, in
     return e == cudaSuccess ? TTF_OK : cuda_fail(e);
 }
 
+int ttf_profile_read_floor(const void* const* buffers, int nbuffers, size_t bytes, int reps, double* ms_per_launch,
+                           ttf_stream_t stream) {
+    if (!buffers || nbuffers < 1 || bytes < 16 || bytes % 16 != 0 || reps < 1 || !ms_per_launch) return TTF_ERR_INVALID_ARG;
+    for (int n = 0; n < nbuffers; ++n)
+        if (!buffers[n] || reinterpret_cast<uintptr_t>(buffers[n]) % 16 != 0) return TTF_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return cuda_fail(cudaGetLastError());
+    cudaError_t e = cudaSuccess;
+    for (int n = 0; n < nbuffers && e == cudaSuccess; ++n) e = launch_read_floor(buffers[n], bytes, nullptr, st);   // warm-up
+    cudaEventRecord(e0, st);
+    for (int rep = 0; rep < reps && e == cudaSuccess; ++rep)
+        for (int n = 0; n < nbuffers && e == cudaSuccess; ++n) e = launch_read_floor(buffers[n], bytes, nullptr, st);
+    cudaEventRecord(e1, st);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    *ms_per_launch = (double)ms / ((double)reps * (double)nbuffers);
+    return e == cudaSuccess ? TTF_OK : cuda_fail(e);
+}
+
 int ttf_release(void) {
     std::lock_guard<std::mutex> lk(g_mu);
     int cur = 0;

@@ -202,4 +202,30 @@ cudaError_t launch_stats(const float* sim, const unsigned char* keep, const int*
     return cudaGetLastError();
 }
 
+// Measurement aid: the plainest kernel that reads a buffer once (fully coalesced, eight 16-byte loads in flight per
+// thread, eight CTAs of 256 threads per SM, launched like the kernels of the pass).  What a launch of this kind
+// takes on one clip is the floor for any kernel that must read that clip: ramp-up and tail of a launch that lasts
+// some 10 us are a visible share of it, so it is well below the copy rate of large buffers.
+__global__ void __launch_bounds__(kXThreads)
+k_read_floor(const uint4* __restrict__ buf, long long n16, unsigned* __restrict__ sink)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    unsigned acc = 0;
+    const long long stride = (long long)gridDim.x * kXThreads * 8;
+    for (long long i0 = (long long)blockIdx.x * kXThreads * 8 + threadIdx.x; i0 < n16; i0 += stride) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = i0 + u * kXThreads < n16 ? __ldcs(buf + i0 + u * kXThreads) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) acc += v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+    }
+    if (acc == 0x9e3779b9u && sink) *sink = acc;       // keeps the loads alive; practically never true
+}
+
+cudaError_t launch_read_floor(const void* buf, size_t bytes, unsigned* sink, cudaStream_t st) {
+    return launch_pdl(k_read_floor, dim3((unsigned)(8 * sm_count())), dim3(kXThreads), st,
+                      reinterpret_cast<const uint4*>(buf), (long long)(bytes / 16), sink);
+}
+
 }  // namespace ttf

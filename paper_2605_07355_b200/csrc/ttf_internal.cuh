@@ -114,6 +114,7 @@ cudaError_t launch_restore(const void* comp, size_t row_bytes, int F, int N, con
                            cudaStream_t st);
 cudaError_t launch_sim_histogram(const float* sim, const int* anchor, int F, int N, int bins, unsigned int* hist,
                                  cudaStream_t st);
+cudaError_t launch_read_floor(const void* buf, size_t bytes, unsigned* sink, cudaStream_t st);
 cudaError_t launch_stats(const float* sim, const unsigned char* keep, const int* anchor, int F, int N, float t, float band,
                          long long* out, cudaStream_t st);
 

@@ -115,6 +115,10 @@ def test_batch_and_variant_entry_points_validate_before_any_cuda_call(lib):
     assert lib.ttf_stats(fake, fake, fake, 4, 4, 4, 0.7, -1.0, fake, None) == 1                  # negative band
     assert lib.ttf_stats(fake, fake, fake, 4, 4, 4, float("nan"), 1e-4, fake, None) == 1
     assert lib.ttf_stats(fake, fake, fake, 0, 4, 4, 0.7, 1e-4, fake, None) == 1
+    one = ctypes.c_double()
+    assert lib.ttf_profile_read_floor(arr, 2, ctypes.c_size_t(24), 1, ctypes.byref(one), None) == 1     # not a multiple of 16
+    assert lib.ttf_profile_read_floor(hole, 2, ctypes.c_size_t(32), 1, ctypes.byref(one), None) == 1
+    assert lib.ttf_profile_read_floor(arr, 2, ctypes.c_size_t(32), 0, ctypes.byref(one), None) == 1
     assert lib.ttf_set_schedule(9) == 1 and lib.ttf_set_schedule(-1) == 1
     assert lib.ttf_set_schedule(0) == 0
 
