@@ -154,7 +154,7 @@ static int make_problem(const void* X, int F, int H, int W, int C, int r, float 
     p->use_tc = 0;
     const int which = g_match_kernel.load();
     if (tc_match_eligible(*p)) p->use_tc = which == 2 || (which == 0 && (r == 2 || tc_match_pieces(*p) == 1)) ? 1 : 0;
-    p->chain = 0; p->chain_next = 0;
+    p->chain = 0; p->chain_next = 0; p->overlapped = 0;
     return TTF_OK;
 }
 
@@ -624,6 +624,7 @@ static int batch_on_streams(const void* const* features, int nclips, int F, int 
     for (int n = 0; n < nclips && first_rc == TTF_OK; ++n) {
         const int lane = n % lanes, turn = n / lanes;
         void* block = (char*)ws[lane] + (size_t)(turn & 1) * stride;
+        ps[n].overlapped = lanes;
         ps[n].chain = turn > 0 ? 1 : 0;          // the lane's previous kernel is the gather of its previous clip
         if (turn < 2) {
             // the block may hold anything (another shape's data, or a failed call's counters): clear its control words
@@ -954,9 +955,12 @@ int ttf_profile_stages(const void* const* features, int nclips, int F, int H, in
         if (!features[n] || !out_tokens[n] || !out_count[n] || !out_pos_thw[n]) return TTF_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     std::vector<Problem> ps(nclips);
+    int want = g_sched_lanes.load();             // the kernels a batch call of these clips would launch
+    if (want < 1 || want > kBatchStreams) want = kBatchStreams;
     for (int n = 0; n < nclips; ++n) {
         int rc = make_problem(features[n], F, H, W, C, r, t, dtype, &ps[n]);
         if (rc != TTF_OK) return rc;
+        ps[n].overlapped = nclips < want ? nclips : want;
     }
     Scratch s0;
     carve_scratch(ps[0], nullptr, &s0);

@@ -47,6 +47,7 @@ struct Problem {
     int chain;          // 1: the kernel before this call's sweep in the stream is the gather of the library's previous
                         // clip, which works on another scratch block: the sweep may run beside it
     int chain_next;     // 1: the kernel after this call's gather is such a sweep
+    int overlapped;     // clips whose kernels run beside one another: the lanes of a batch (0 or 1: this call runs alone)
 };
 
 // Device pointers carved out of one scratch allocation.
