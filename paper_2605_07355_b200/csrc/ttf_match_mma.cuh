@@ -226,6 +226,7 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
         mma_consume_stage<MT, NT, GRAM>(wring + (b % kMmaStages) * PIECES * 32, lane, acc, accn, accb);
     }
     cp_async_wait<0>();
+    pdl_launch_dependents();                     // (here rather than at the start: see match_mma_body)
     __syncthreads();                             // every warp is done with its ring: reuse it for the partials
 
     // accumulator fragment: c0,c1 = (frame g, candidates 2*tig, 2*tig+1); c2,c3 = (frame g+8, same candidates)
