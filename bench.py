@@ -43,7 +43,7 @@ def parse_args():
     ap.add_argument("--streams", type=int, default=0,
                     help="0: one ttf_compress_batch call per step (the library spreads the clips over its own "
                          "streams, see --lanes); S > 0: one ttf_compress call per clip on S streams of the caller")
-    ap.add_argument("--lanes", type=int, default=0, help="clips of a batch in flight (ttf_set_schedule); 0 = automatic")
+    ap.add_argument("--lanes", type=int, default=0, help="clips of a batch in flight (ttf_set_schedule); 0 = automatic, -1 = the pipelined schedule")
     ap.add_argument("--match-kernel", default="auto", choices=["auto", "mma", "tc"],
                     help="kernel of the matching step for bf16 clips (ttf_set_match_kernel)")
     ap.add_argument("--threshold", type=float, default=None)
@@ -385,7 +385,7 @@ def main():
     amode = {"auto": 0, "first": 1, "last": 2}[args.anchor]
     P.ttf_set_match_kernel({"auto": 0, "mma": 1, "tc": 2}[args.match_kernel])
     P.ttf_set_schedule(args.lanes)
-    lanes = args.lanes if args.lanes > 0 else 8
+    lanes = args.lanes if args.lanes > 0 else ("2, pipelined" if args.lanes == -1 and amode == 0 else 8)
 
     def step():
         if args.streams == 0:

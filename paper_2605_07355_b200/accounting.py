@@ -42,7 +42,7 @@ def kernel_bytes(kind: str, F: int, N: int, C: int, itemsize: int, count: int) -
     raise KeyError(kind)
 
 
-def pipeline_dram_bytes_model(F: int, N: int, C: int, itemsize: int, count: int, lanes: int, fixed_anchor: bool = False) -> int:
+def pipeline_dram_bytes_model(F: int, N: int, C: int, itemsize: int, count: int, lanes, fixed_anchor: bool = False) -> int:
     """DRAM bytes one clip moves in the pipeline as scheduled (confirmed with the profiler's DRAM counters over a
     whole step: 93.8 / 153.4 / 172.7 MB per 8B-shaped clip for 1 / 2 / 8 clips in flight, 113.7 MB with a fixed
     anchor).  With one clip in flight the matching pass and the gather find the clip in L2, so it is read once; with
@@ -52,6 +52,8 @@ def pipeline_dram_bytes_model(F: int, N: int, C: int, itemsize: int, count: int,
     X = F * N * C * itemsize
     rows = count * C * itemsize
     small = F * N * 9 + count * 12 + 4
+    if lanes == "2, pipelined":         # X once, the kept rows for the gather again, the output (measured: 133 MB,
+        return X + 2 * rows + small     # the model's 114 MB plus what the matching pass still misses)
     if lanes <= 1:
         return X + rows + small
     return (1 if fixed_anchor else 2) * X + 2 * rows + small

@@ -28,6 +28,7 @@ EXPORTS = [
 TTF_ERR_TIMEOUT, TTF_ERR_STATIC_LIMIT, TTF_ERR_BOUNDS = 5, 6, 7
 TTF_ANCHOR_AUTO, TTF_ANCHOR_FIRST, TTF_ANCHOR_LAST, TTF_ANCHOR_EXPLICIT = 0, 1, 2, 3
 TTF_ORDER_ANCHOR_FIRST, TTF_ORDER_NATURAL = 0, 1
+TTF_SCHEDULE_PIPELINED = -1
 
 
 class TTFOptions(ctypes.Structure):
@@ -273,7 +274,8 @@ def ttf_set_match_kernel(which: int = 0) -> None:
 
 
 def ttf_set_schedule(clips_in_flight: int = 0) -> None:
-    """ttf_set_schedule: clips of a batch in flight (0 = automatic)."""
+    """ttf_set_schedule: clips of a batch in flight (0 = automatic, 1 to 8, or TTF_SCHEDULE_PIPELINED = -1: two
+    lanes in opposite phases with the matching pass served by L2)."""
     rc = lib().ttf_set_schedule(int(clips_in_flight))
     if rc != TTF_OK:
         raise TTFError(rc, "ttf_set_schedule")

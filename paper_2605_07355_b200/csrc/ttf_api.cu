@@ -154,7 +154,7 @@ static int make_problem(const void* X, int F, int H, int W, int C, int r, float 
     p->use_tc = 0;
     const int which = g_match_kernel.load();
     if (tc_match_eligible(*p)) p->use_tc = which == 2 || (which == 0 && (r == 2 || tc_match_pieces(*p) == 1)) ? 1 : 0;
-    p->chain = 0; p->chain_next = 0; p->overlapped = 0;
+    p->chain = 0; p->chain_next = 0; p->overlapped = 0; p->stream_once = 0;
     return TTF_OK;
 }
 
@@ -566,7 +566,12 @@ int ttf_compress_mean(const void* features, int F, int H, int W, int C, int r, f
 // and drain, so a batch is spread round-robin over kBatchStreams internal streams per device that fork from the
 // caller's stream and join it again (events only: the call stays asynchronous and can be captured in a graph).
 constexpr int kBatchStreams = 8;
-struct BatchLanes { cudaStream_t s[kBatchStreams] = {}; cudaEvent_t fork = nullptr; cudaEvent_t join[kBatchStreams] = {}; bool ok = false; };
+constexpr int kMatchedRing = 4;                  // events "clip n has been matched" of the pipelined schedule, used in turn
+struct BatchLanes {
+    cudaStream_t s[kBatchStreams] = {}; cudaEvent_t fork = nullptr; cudaEvent_t join[kBatchStreams] = {};
+    cudaEvent_t matched[kMatchedRing] = {};
+    bool ok = false;
+};
 static std::map<int, BatchLanes> g_lanes;
 static std::mutex g_lane_mu;                     // the fork / join events are shared: one batch is enqueued at a time
 
@@ -582,6 +587,8 @@ static int batch_lanes(BatchLanes** out) {
             e = cudaStreamCreateWithFlags(&L.s[i], cudaStreamNonBlocking);
             if (e == cudaSuccess) e = cudaEventCreateWithFlags(&L.join[i], cudaEventDisableTiming);
         }
+        for (int i = 0; i < kMatchedRing && e == cudaSuccess; ++i)
+            e = cudaEventCreateWithFlags(&L.matched[i], cudaEventDisableTiming);
         if (e != cudaSuccess) return cuda_fail(e);
         L.ok = true;
     }
@@ -609,6 +616,15 @@ static int batch_on_streams(const void* const* features, int nclips, int F, int 
         if (s.bytes > stride) stride = s.bytes;
     }
     int want = g_sched_lanes.load();
+    // Pipelined schedule (TTF_SCHEDULE_PIPELINED, automatic anchor only).  Eq. (auto_anchor) forces two passes over X;
+    // the second is free only while the clip is still in L2, which holds one 8B-shaped clip and most of a second.
+    // Two lanes in opposite phases: the matching kernels of consecutive clips are ordered one after the other, and a
+    // lane's next sweep starts when its previous clip has been matched (the chain below), so at any time one clip is
+    // matched out of L2 while the next one streams in.  The matching kernel marks the source rows it has read, and
+    // the gather what it reads and writes, as the first lines to leave L2; without that the incoming clip displaces
+    // exactly the rows that are still to be matched (they are the oldest lines).
+    const bool pipelined = want == TTF_SCHEDULE_PIPELINED && nclips >= 3 && ps[0].anchor_mode == 0;
+    if (pipelined) want = 2;
     if (want < 1 || want > kBatchStreams) want = kBatchStreams;      // automatic: measured best for every clip shape so far
     const int lanes = nclips < want ? nclips : want;
     std::vector<void*> ws(lanes, nullptr);
@@ -625,6 +641,7 @@ static int batch_on_streams(const void* const* features, int nclips, int F, int 
         const int lane = n % lanes, turn = n / lanes;
         void* block = (char*)ws[lane] + (size_t)(turn & 1) * stride;
         ps[n].overlapped = lanes;
+        ps[n].stream_once = pipelined ? 1 : 0;
         ps[n].chain = turn > 0 ? 1 : 0;          // the lane's previous kernel is the gather of its previous clip
         if (turn < 2) {
             // the block may hold anything (another shape's data, or a failed call's counters): clear its control words
@@ -635,7 +652,22 @@ static int batch_on_streams(const void* const* features, int nclips, int F, int 
         }
         // (the lane's next clip, if there is one, is at turn + 1; its sweep is chained from turn 2 on)
         ps[n].chain_next = (n + lanes < nclips && turn + 1 >= 2) ? 1 : 0;
-        first_rc = compress_impl(ps[n], block, out_tokens[n], out_count[n], out_pos_thw[n], L->s[lane]);
+        if (!pipelined) {
+            first_rc = compress_impl(ps[n], block, out_tokens[n], out_count[n], out_pos_thw[n], L->s[lane]);
+            continue;
+        }
+        // the same kernels as compress_impl, with the matching kernel ordered after that of the clip before (which
+        // ran in the other lane)
+        Scratch sc;
+        carve_scratch(ps[n], block, &sc);
+        cudaStream_t ls = L->s[lane];
+        { ProfScope pr(ls, PK_NORM_SUM); e = launch_norm_sum(ps[n], sc, ls); }
+        if (e == cudaSuccess) { ProfScope pr(ls, PK_FRAME_STATS); e = launch_frame_stats(ps[n], sc, nullptr, ls); }
+        if (e == cudaSuccess && n > 0) e = cudaStreamWaitEvent(ls, L->matched[(n - 1) % kMatchedRing], 0);
+        if (e == cudaSuccess) { ProfScope pr(ls, PK_MATCH); e = launch_match(ps[n], sc, nullptr, sc.shat, sc.dst, sc.keep, ls); }
+        if (e == cudaSuccess) e = cudaEventRecord(L->matched[n % kMatchedRing], ls);
+        if (e == cudaSuccess) { ProfScope pr(ls, PK_COMPACT); e = launch_compact(ps[n], sc, out_tokens[n], out_pos_thw[n], out_count[n], ls); }
+        if (e != cudaSuccess) first_rc = cuda_fail(e);
     }
     {   // the caller asks about the batch through its own stream: point it at the lanes' error words
         int dev = 0;
@@ -661,7 +693,7 @@ int ttf_set_match_kernel(int which) {
 }
 
 int ttf_set_schedule(int clips_in_flight) {
-    if (clips_in_flight < 0 || clips_in_flight > kBatchStreams) return TTF_ERR_INVALID_ARG;
+    if (clips_in_flight < TTF_SCHEDULE_PIPELINED || clips_in_flight > kBatchStreams) return TTF_ERR_INVALID_ARG;
     g_sched_lanes.store(clips_in_flight);
     return TTF_OK;
 }

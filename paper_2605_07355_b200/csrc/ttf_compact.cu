@@ -80,7 +80,7 @@ k_compact_bulk(const unsigned char* __restrict__ X, size_t row_bytes, int F, int
                const unsigned char* __restrict__ keep, const int* __restrict__ dst,
                unsigned char* __restrict__ out_tokens, int* __restrict__ out_pos, int* __restrict__ out_count,
                int* __restrict__ fuse_cnt, int ncopy_blocks, int NA, int acnt, int t_off, int pos_base,
-               int late_trigger, int wait_limit, int tx_extra)
+               int late_trigger, int wait_limit, int tx_extra, int stream_once)
 {
     extern __shared__ __align__(128) unsigned char stage[];     // [kCopyWarps][kBulkPiece]
     __shared__ uint64_t bar[kCopyWarps];
@@ -115,6 +115,9 @@ k_compact_bulk(const unsigned char* __restrict__ X, size_t row_bytes, int F, int
     const int pieces = (int)((row_bytes + kBulkPiece - 1) / kBulkPiece);
     uint32_t phase = 0;
     bool gave_up = false;
+    // pipelined schedule: neither the rows read here nor the rows written are needed in L2 again, while the clip
+    // that is being matched and the one streaming in are: their lines are the first to go
+    const unsigned long long once = l2_evict_first_policy();
     for (int j = gw; ; j += nw) {
         int f;
         if (j < NA) f = a * N + j;               // anchor rows first (Eq. xprime_stack)
@@ -138,14 +141,16 @@ k_compact_bulk(const unsigned char* __restrict__ X, size_t row_bytes, int F, int
                 const uint32_t bytes = (uint32_t)(row_bytes - off < (size_t)kBulkPiece ? row_bytes - off : kBulkPiece);
                 bulk_wait_read<0>();             // the previous store has finished reading the buffer
                 mbar_arrive_expect_tx(&bar[w], bytes + (uint32_t)tx_extra);
-                bulk_load(buf, X + (size_t)f * row_bytes + off, bytes, &bar[w]);
+                if (stream_once) bulk_load_hint(buf, X + (size_t)f * row_bytes + off, bytes, &bar[w], once);
+                else bulk_load(buf, X + (size_t)f * row_bytes + off, bytes, &bar[w]);
                 if (!mbar_wait(&bar[w], phase & 1, wait_limit)) {
                     mbar_wait(&bar[w], phase & 1, wait_limit);   // one more bounded chance for the copy to land
                     gave_up = true;
                     break;
                 }
                 ++phase;
-                bulk_store(out_tokens + (size_t)j * row_bytes + off, buf, bytes);
+                if (stream_once) bulk_store_hint(out_tokens + (size_t)j * row_bytes + off, buf, bytes, once);
+                else bulk_store(out_tokens + (size_t)j * row_bytes + off, buf, bytes);
                 bulk_commit();
             }
         }
@@ -278,7 +283,7 @@ cudaError_t launch_compact(const Problem& p, const Scratch& s, void* out_tokens,
         return launch_ex(pdl, smem, k_compact_bulk, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, s.hdr,
                          (const int*)s.cnt, (const int*)s.prefix, (const unsigned char*)s.keep, (const int*)s.dst, out,
                          out_pos, out_count, s.fuse_cnt, ncopy, NA, acnt, p.pos_t_offset, p.pos_base, p.chain_next,
-                         wait_poll_limit(), wait_tx_extra());
+                         wait_poll_limit(), wait_tx_extra(), p.stream_once);
     }
     if (esize == 4)
         return launch_pdl_if(pdl, k_compact<4>, g, b, st, X, row_bytes, p.F, p.H, p.W, p.r, (const int*)s.hdr,

@@ -48,6 +48,8 @@ struct Problem {
                         // clip, which works on another scratch block: the sweep may run beside it
     int chain_next;     // 1: the kernel after this call's gather is such a sweep
     int overlapped;     // clips whose kernels run beside one another: the lanes of a batch (0 or 1: this call runs alone)
+    int stream_once;    // 1: the matching kernel marks the lines of the source rows it reads as the first to leave L2
+                        // (the pipelined schedule: the next clip streams into L2 while this one is matched)
 };
 
 // Device pointers carved out of one scratch allocation.
@@ -179,6 +181,12 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, c
 
 // griddepcontrol: wait = all kernels this one depends on have completed and their writes are visible (a no-op
 // for a normally launched kernel); launch_dependents = the next kernel of the stream may be scheduled.
+// L2 cache policy for data that is read once more and then dead: its lines are evicted before any others
+__device__ __forceinline__ unsigned long long l2_evict_first_policy() {
+    unsigned long long pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 

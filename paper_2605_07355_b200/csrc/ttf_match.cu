@@ -93,7 +93,8 @@ template <int MT, int NT, bool GRAM, int ST>
 __device__ __forceinline__ void match_mma_body(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t,
                                                const AnchorSrc& asrc, const float* ssq, int nslice,
                                                float* __restrict__ shat, int* __restrict__ dst,
-                                               unsigned char* __restrict__ keep, int* __restrict__ cnt)
+                                               unsigned char* __restrict__ keep, int* __restrict__ cnt,
+                                               int stream_once)
 {
     extern __shared__ __align__(128) unsigned char dyn_smem[];
     const int N = H * W;
@@ -119,7 +120,7 @@ __device__ __forceinline__ void match_mma_body(const bf16_t* __restrict__ X, int
         trace_mark(asrc.hdr, 4, true);
         return a;
     };
-    match_mma_unit<MT, NT, GRAM, ST>(X, F, H, W, C, r, t, anchor_fn, i, k0, ssq, nslice, shat, dst, keep, cnt, asrc.hdr, dyn_smem);
+    match_mma_unit<MT, NT, GRAM, ST>(X, F, H, W, C, r, t, anchor_fn, i, k0, ssq, nslice, shat, dst, keep, cnt, asrc.hdr, dyn_smem, stream_once);
     trace_mark(asrc.hdr, 2, true);
 }
 
@@ -127,9 +128,10 @@ __device__ __forceinline__ void match_mma_body(const bf16_t* __restrict__ X, int
 template <int MT, int NT>
 __global__ void TTF_MMA_BOUNDS
 k_match_mma(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r, float t, AnchorSrc asrc,
-            float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt)
+            float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt,
+            int stream_once)
 {
-    match_mma_body<MT, NT, true, kMmaStagesDefault>(X, F, H, W, C, r, t, asrc, nullptr, 0, shat, dst, keep, cnt);
+    match_mma_body<MT, NT, true, kMmaStagesDefault>(X, F, H, W, C, r, t, asrc, nullptr, 0, shat, dst, keep, cnt, stream_once);
 }
 
 // r = 2: the 25 candidate rows of a cell are as much data as 25 source rows, so a CTA takes 64 frames per cell to
@@ -142,7 +144,7 @@ k_match_mma_wide(const bf16_t* __restrict__ X, int F, int H, int W, int C, int r
                  const float* __restrict__ ssq, int nslice,
                  float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt)
 {
-    match_mma_body<kWideMT, 4, false, kWideStages>(X, F, H, W, C, r, t, asrc, ssq, nslice, shat, dst, keep, cnt);
+    match_mma_body<kWideMT, 4, false, kWideStages>(X, F, H, W, C, r, t, asrc, ssq, nslice, shat, dst, keep, cnt, 0);
 }
 
 template <int MT, int NT>
@@ -154,7 +156,7 @@ static cudaError_t launch_mma_t(const Problem& p, const Scratch& s, int* out_anc
     if (e != cudaSuccess) return e;
     return launch_ex(true, smem, k_match_mma<MT, NT>, dim3((unsigned)(chunks * p.N)),
                      dim3(kMmaWarps * 32), st, reinterpret_cast<const bf16_t*>(p.X), p.F, p.H, p.W, p.C, p.r, p.t,
-                     make_anchor_src(p, s, out_anchor), shat, dst, keep, s.cnt);
+                     make_anchor_src(p, s, out_anchor), shat, dst, keep, s.cnt, p.stream_once);
 }
 
 static cudaError_t launch_mma_wide(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,

@@ -44,6 +44,12 @@ __device__ __forceinline__ void cp_async16(void* dst_smem, const void* src, bool
     const int bytes = valid ? 16 : 0;            // 0 source bytes: the 16 destination bytes are zero-filled
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
 }
+// the same copy with an L2 cache policy (createpolicy) on the line it reads
+__device__ __forceinline__ void cp_async16_hint(void* dst_smem, const void* src, bool valid, unsigned long long policy) {
+    const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(dst_smem));
+    const int bytes = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2, %3;" ::"r"(d), "l"(src), "r"(bytes), "l"(policy) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
@@ -52,14 +58,23 @@ template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile(
 template <int MT, int NT, bool DO_A = true, bool DO_B = true>
 __device__ __forceinline__ void mma_issue_stage(uint4* slot, const uint4* const (&arow)[MT][2],
                                                 const uint4* const (&brow)[NT], const bool (&bvalid)[NT],
-                                                int idx, int units, int lane) {
+                                                int idx, int units, int lane, int stream_once) {
     const bool ok = idx < units;
     const int safe = ok ? idx : 0;
     if constexpr (DO_A) {
+        // a source row is read by this CTA alone: where the next clip streams into L2 meanwhile, its lines go first
+        if (stream_once) {
+            const unsigned long long once = l2_evict_first_policy();
 #pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
+            for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-            for (int h = 0; h < 2; ++h) cp_async16(slot + (mt * 2 + h) * 32 + lane, arow[mt][h] + safe, ok);
+                for (int h = 0; h < 2; ++h) cp_async16_hint(slot + (mt * 2 + h) * 32 + lane, arow[mt][h] + safe, ok, once);
+        } else {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) cp_async16(slot + (mt * 2 + h) * 32 + lane, arow[mt][h] + safe, ok);
+        }
     }
     if constexpr (DO_B) {
 #pragma unroll
@@ -120,7 +135,7 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
                                                AnchorFn anchor_fn, int i, int k0, const float* ssq, int nslice,
                                                float* __restrict__ shat, int* __restrict__ dst,
                                                unsigned char* __restrict__ keep, int* __restrict__ cnt,
-                                               int* hdr, unsigned char* dyn_smem)
+                                               int* hdr, unsigned char* dyn_smem, int stream_once)
 {
     constexpr int kMmaStages = ST;
     constexpr int FR = 16 * MT;      // frames per CTA
@@ -174,7 +189,7 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
     for (int st = 0; st < kMmaStages - 1; ++st)
         if (st < nmine)
             mma_issue_stage<MT, NT, true, false>(wring + st * PIECES * 32, arow, brow, bvalid,
-                                                 (w + st * kMmaWarps) * 4 + tig, units, lane);
+                                                 (w + st * kMmaWarps) * 4 + tig, units, lane, stream_once);
     cp_async_commit();
 
     const int a = anchor_fn();
@@ -213,14 +228,14 @@ __device__ __forceinline__ void match_mma_unit(const bf16_t* __restrict__ X, int
     for (int st = 0; st < kMmaStages - 1; ++st) {
         if (st < nmine)
             mma_issue_stage<MT, NT, false, true>(wring + st * PIECES * 32, arow, brow, bvalid,
-                                                 (w + st * kMmaWarps) * 4 + tig, units, lane);
+                                                 (w + st * kMmaWarps) * 4 + tig, units, lane, stream_once);
         cp_async_commit();
     }
     for (int b = 0; b < nmine; ++b) {
         const int nb = b + kMmaStages - 1;
         if (nb < nmine)
             mma_issue_stage<MT, NT>(wring + (nb % kMmaStages) * PIECES * 32, arow, brow, bvalid,
-                                    (w + nb * kMmaWarps) * 4 + tig, units, lane);
+                                    (w + nb * kMmaWarps) * 4 + tig, units, lane, stream_once);
         cp_async_commit();
         cp_async_wait<kMmaStages - 1>();         // block b has landed (each lane waits for its own copies)
         mma_consume_stage<MT, NT, GRAM>(wring + (b % kMmaStages) * PIECES * 32, lane, acc, accn, accb);

@@ -52,6 +52,15 @@ __device__ __forceinline__ void tma_load_4d(void* dst_smem, const CUtensorMap* m
           "r"(smem_u32(bar))
         : "memory");
 }
+// the same copy with an L2 cache policy (createpolicy) on the lines it reads
+__device__ __forceinline__ void tma_load_4d_hint(void* dst_smem, const CUtensorMap* map, int c0, int c1, int c2, int c3,
+                                                 uint64_t* bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3, %4, %5}], [%6], %7;"
+        ::"r"(smem_u32(dst_smem)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
+          "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
 __device__ __forceinline__ void tensormap_prefetch(const CUtensorMap* map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -155,7 +164,7 @@ __global__ void __launch_bounds__(kTcThreads)
 k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
            int F, int H, int W, int C, float t, AnchorSrc asrc, int pieces,
            float* __restrict__ shat, int* __restrict__ dst, unsigned char* __restrict__ keep, int* __restrict__ cnt,
-           int wait_limit, int tx_extra)
+           int wait_limit, int tx_extra, int stream_once)
 {
     using S = TcShape<R>;
     extern __shared__ unsigned char dyn_raw[];
@@ -226,6 +235,7 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
         // ---- producer: one lane issues the tile copies of every stage ----------------------------------------
         if (lane == 0) {
             int issued = 0;
+            const uint64_t once = l2_evict_first_policy();
             for (int it = 0; it < nst; ++it) {
                 const int s = it % S::STAGES;
                 if (it >= S::STAGES && !mbar_wait(&bar_empty[s], ((it / S::STAGES) & 1) ^ 1, wait_limit)) { atomicExch(&s_err, 1); break; }
@@ -233,7 +243,10 @@ k_match_tc(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUt
                 unsigned char* sa = dyn + (size_t)s * S::STAGE;
                 const int c0 = (st0 + it) * kTcKC;
                 mbar_arrive_expect_tx(&bar_full[s], kTcABytes + S::BBOX + (uint32_t)tx_extra);   // (extra: test hook only)
-                tma_load_4d(sa, &mapA, c0, x0, y, k0, &bar_full[s]);
+                // source rows are read by this tile alone: in a schedule that streams the next clip into L2 meanwhile,
+                // their lines are the ones to give up first (the candidate rows are shared with neighbouring tiles)
+                if (stream_once) tma_load_4d_hint(sa, &mapA, c0, x0, y, k0, &bar_full[s], once);
+                else tma_load_4d(sa, &mapA, c0, x0, y, k0, &bar_full[s]);
                 tma_load_4d(sa + kTcABytes, &mapB, c0, x0 - R, y - R, a, &bar_full[s]);
                 issued = it + 1;
             }
@@ -486,7 +499,7 @@ static cudaError_t launch_tc_t(const Problem& p, const Scratch& s, int* out_anch
     }
     cfg.attrs = attr; cfg.numAttrs = n;
     return cudaLaunchKernelEx(&cfg, k_match_tc<R>, mapA, mapB, p.F, p.H, p.W, p.C, p.t, make_anchor_src(p, s, out_anchor),
-                              pieces, shat, dst, keep, s.cnt, wait_poll_limit(), wait_tx_extra());
+                              pieces, shat, dst, keep, s.cnt, wait_poll_limit(), wait_tx_extra(), p.stream_once);
 }
 
 cudaError_t launch_match_tc(const Problem& p, const Scratch& s, int* out_anchor, float* shat, int* dst,

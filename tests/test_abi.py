@@ -119,7 +119,8 @@ def test_batch_and_variant_entry_points_validate_before_any_cuda_call(lib):
     assert lib.ttf_profile_read_floor(arr, 2, ctypes.c_size_t(24), 1, ctypes.byref(one), None) == 1     # not a multiple of 16
     assert lib.ttf_profile_read_floor(hole, 2, ctypes.c_size_t(32), 1, ctypes.byref(one), None) == 1
     assert lib.ttf_profile_read_floor(arr, 2, ctypes.c_size_t(32), 0, ctypes.byref(one), None) == 1
-    assert lib.ttf_set_schedule(9) == 1 and lib.ttf_set_schedule(-1) == 1
+    assert lib.ttf_set_schedule(9) == 1 and lib.ttf_set_schedule(-2) == 1
+    assert lib.ttf_set_schedule(-1) == 0         # TTF_SCHEDULE_PIPELINED
     assert lib.ttf_set_schedule(0) == 0
 
 

@@ -197,3 +197,46 @@ def test_multi_block_scratch_after_another_shape_on_the_same_stream():
         L = int(ref[j][1].item())
         assert int(cnts[j].item()) == L
         assert torch.equal(toks[j][:L], ref[j][0][:L]) and torch.equal(poss[j][:L], ref[j][2][:L])
+
+
+@pytest.mark.parametrize("match_kernel", [1, 2])
+def test_pipelined_schedule_gives_the_same_results(match_kernel):
+    """ttf_set_schedule(TTF_SCHEDULE_PIPELINED): two lanes in opposite phases, L2 eviction hints on the matching
+    pass and the gather; scheduling and cache policy only, so every clip must come out bit for bit as from
+    ttf_compress, and equal to the oracle (8B-shaped clips, seven of them: several turns per lane and a ragged
+    end; then small fp32 clips, which take the kernels without hints)"""
+    s = clips.CONFIGS["vl8b_cal"]
+    Xn = [clips.make_clip(s, s.seed + j) for j in range(7)]
+    Xs = [to_device(x) for x in Xn]
+    P.ttf_set_match_kernel(match_kernel)
+    P.ttf_set_schedule(P.TTF_SCHEDULE_PIPELINED)
+    try:
+        for _ in range(2):                       # the second call finds the scratch blocks as the first left them
+            outs = P.ttf_compress_batch(Xs, s.r, s.t)
+            torch.cuda.synchronize()
+            assert P.ttf_last_device_status() == P.TTF_OK
+            assert_same_as_single(Xs, s.r, s.t, outs)
+        R = O.compress(Xn[5], s.r, s.t)
+        q = P.ttf_query(Xs[5], s.r, s.t)
+        keep = q["keep"].cpu().numpy()
+        assert int(q["anchor"].item()) == R.anchor
+        in_band = np.abs(R.s_hat.astype(np.float32) - np.float32(s.t)) < 1e-4
+        assert not ((keep != R.keep) & ~in_band).any()
+        forced = O.compress(Xn[5], s.r, s.t, anchor_frame=R.anchor, forced_keep=keep)
+        L = int(outs[1][5].item())
+        assert L == forced.count
+        assert (outs[2][5][:L].cpu().numpy() == forced.pos).all() and (to_bits(outs[0][5][:L]) == forced.tokens).all()
+        small = [to_device(corr_clip(5, 4, 5, 40, seed=77 + j, dtype="f32")) for j in range(5)]
+        outs = P.ttf_compress_batch(small, 1, 0.7)
+        torch.cuda.synchronize()
+        assert_same_as_single(small, 1, 0.7, outs)
+        first = P.ttf_compress_batch(Xs[:4], s.r, s.t, anchor_mode=P.TTF_ANCHOR_FIRST)   # fixed anchor: ordinary lanes
+        torch.cuda.synchronize()
+        for j in range(4):
+            a = P.ttf_compress(Xs[j], s.r, s.t, anchor_mode=P.TTF_ANCHOR_FIRST)
+            torch.cuda.synchronize()
+            L = int(a[1].item())
+            assert int(first[1][j].item()) == L and torch.equal(first[0][j][:L], a[0][:L])
+    finally:
+        P.ttf_set_schedule(0)
+        P.ttf_set_match_kernel(0)
