@@ -139,6 +139,21 @@ def test_bench_configuration_full_size_against_oracle():
         assert (to_bits(toks[j][:L]) == forced.tokens).all()
         rhos.append(1.0 - L / s.tokens)
     assert abs(float(np.mean(rhos)) - 0.67) < 0.03
+    # the benchmark replays the call from a CUDA graph: the replayed batch must write the same bytes
+    st = torch.cuda.Stream()
+    gt = [torch.zeros_like(x) for x in toks]
+    gc = [torch.zeros_like(x) for x in cnts]
+    gp = [torch.zeros_like(x) for x in poss]
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=st):
+        P.ttf_compress_batch(Xs, s.r, s.t, gt, gc, gp, stream=st)
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize()
+    for j in range(n):
+        L = int(cnts[j].item())
+        assert int(gc[j].item()) == L
+        assert torch.equal(gt[j][:L], toks[j][:L]) and torch.equal(gp[j][:L], poss[j][:L])
 
 
 def test_host_batch_fp32_and_single_clip():
